@@ -1,0 +1,106 @@
+"""RNN-T model pieces the search calls (Sec. 3.1): joiner j(t,u,k) followed by
+softmax normalisation J, and the prediction network g(u).  fp64 throughout.
+
+Joiner form (synthetic workloads): z = W_out . tanh(W_e h_t + W_p g_u) + b_out.
+Predictor: either stateless (g = embedding of the last token; the empty
+prefix uses the blank token's embedding) or a stack of LSTM layers with gate
+order (input, forget, cell, output) and a single bias per layer, started by
+feeding the blank token from an all-zero state (InitPredictor, Sec. 3.2).
+"""
+from typing import List, Optional, Sequence, Tuple
+
+import numpy as np
+
+
+def _f64(x):
+    return np.asarray(x, dtype=np.float64)
+
+
+class RnntModel:
+    def __init__(self, W_e, W_p, W_out, b_out, emb,
+                 lstm_W_ih: Sequence = (), lstm_W_hh: Sequence = (), lstm_b: Sequence = (),
+                 blank: int = 0):
+        self.W_e = _f64(W_e)        # [J, D_enc]
+        self.W_p = _f64(W_p)        # [J, P]
+        self.W_out = _f64(W_out)    # [V, J]
+        self.b_out = _f64(b_out)    # [V]
+        self.emb = _f64(emb)        # [V, emb_dim]
+        self.lstm_W_ih = [_f64(w) for w in lstm_W_ih]   # [4Hd, in]
+        self.lstm_W_hh = [_f64(w) for w in lstm_W_hh]   # [4Hd, Hd]
+        self.lstm_b = [_f64(b) for b in lstm_b]         # [4Hd]
+        self.blank = int(blank)
+        self.V = self.W_out.shape[0]
+        assert self.W_e.shape[0] == self.W_p.shape[0] == self.W_out.shape[1]
+        assert len(self.lstm_W_ih) == len(self.lstm_W_hh) == len(self.lstm_b)
+
+    @property
+    def is_lstm(self) -> bool:
+        return len(self.lstm_W_ih) > 0
+
+
+def log_softmax(z: np.ndarray) -> np.ndarray:
+    """log J = z - log sum_k exp z_k over the last axis (Sec. 3.1: J is the
+    joiner output after softmax normalisation)."""
+    m = z.max(axis=-1, keepdims=True)
+    return z - (m + np.log(np.exp(z - m).sum(axis=-1, keepdims=True)))
+
+
+def joiner_log_probs(model: RnntModel, seg: np.ndarray, pred_out: np.ndarray) -> np.ndarray:
+    """J = Softmax(Joiner(seg, pred)) of Algorithm 1, in log space.
+
+    seg [S', D_enc] encoder frames, pred_out [H, P] predictor outputs
+    -> log J [H, S', V] for every (hypothesis, frame) pair."""
+    e = _f64(seg) @ model.W_e.T                     # [S', J]
+    p = _f64(pred_out) @ model.W_p.T                # [H, J]
+    hidden = np.tanh(e[None, :, :] + p[:, None, :])  # [H, S', J]
+    z = hidden @ model.W_out.T + model.b_out        # [H, S', V]
+    return log_softmax(z)
+
+
+def _sigmoid(x):
+    return 1.0 / (1.0 + np.exp(-x))
+
+
+PredState = Optional[Tuple[List[np.ndarray], List[np.ndarray]]]
+
+
+def lstm_step(model: RnntModel, state: PredState, token: int):
+    """One predictor step on `token`.  state = (h[l], c[l]) per layer."""
+    h_prev, c_prev = state
+    x = model.emb[token]
+    h_new, c_new = [], []
+    for l in range(len(model.lstm_W_ih)):
+        gates = model.lstm_W_ih[l] @ x + model.lstm_W_hh[l] @ h_prev[l] + model.lstm_b[l]
+        Hd = gates.shape[0] // 4
+        i, f, g, o = (gates[0:Hd], gates[Hd:2 * Hd], gates[2 * Hd:3 * Hd], gates[3 * Hd:4 * Hd])
+        c = _sigmoid(f) * c_prev[l] + _sigmoid(i) * np.tanh(g)
+        h = _sigmoid(o) * np.tanh(c)
+        h_new.append(h)
+        c_new.append(c)
+        x = h
+    return (h_new, c_new), x
+
+
+def predictor_init(model: RnntModel):
+    """InitPredictor(): (state, output) for the empty token prefix."""
+    if not model.is_lstm:
+        return None, model.emb[model.blank].copy()
+    L = len(model.lstm_W_ih)
+    Hd = model.lstm_W_hh[0].shape[1]
+    zero = ([np.zeros(Hd) for _ in range(L)], [np.zeros(Hd) for _ in range(L)])
+    return lstm_step(model, zero, model.blank)
+
+
+def predictor_step(model: RnntModel, state: PredState, token: int):
+    """UpdatePredictorOutput for one hypothesis: (new state, new output)."""
+    if not model.is_lstm:
+        return None, model.emb[token].copy()
+    return lstm_step(model, state, token)
+
+
+def predictor_for_tokens(model: RnntModel, tokens: Sequence[int]):
+    """Predictor output after consuming a whole token prefix."""
+    state, o = predictor_init(model)
+    for k in tokens:
+        state, o = predictor_step(model, state, k)
+    return state, o
