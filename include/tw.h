@@ -1,0 +1,204 @@
+/*
+ * libtw: token-wise beam search for RNN-T (Algorithm 1 of "A Token-Wise Beam
+ * Search Algorithm for RNN-T") on one NVIDIA B200 (sm_100a).
+ *
+ * C ABI.  Conventions that hold for every call unless a comment says otherwise:
+ *   - pointers are DEVICE pointers; a name starting with host_ is a HOST pointer;
+ *   - matrices are dense, row-major, float32; int arrays are int32;
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream);
+ *     work is enqueued on it and the call returns without synchronising, except
+ *     where stated;
+ *   - the caller owns every buffer it passes; the library owns the handle and
+ *     its workspace from tw_init to tw_destroy;
+ *   - every function returns a tw_status; nothing throws, nothing aborts.  A
+ *     failed argument check enqueues no work.
+ *   - scores are natural-log probabilities; log 0 is -infinity.
+ *   - a handle must not be used from two host threads at once, and two calls on
+ *     one handle must not overlap on the GPU (they share its workspace).
+ *
+ * Notation (paper, Sec. 3): T encoder frames, V vocabulary size including the
+ * blank symbol, N beam size, S segment size, J joiner hidden width, P predictor
+ * output width, H <= N live hypotheses of an utterance (list A of Algorithm 1),
+ * R = sum of H over the utterances of a batch ("rows").
+ */
+#ifndef TW_H_
+#define TW_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct tw_handle tw_handle;
+
+typedef enum {
+  TW_OK = 0,
+  TW_ERR_ARG = 1,    /* null pointer, size out of range, inconsistent shapes           */
+  TW_ERR_ALLOC = 2,  /* device or host allocation failed                                */
+  TW_ERR_CUDA = 3,   /* a CUDA call failed; tw_last_cuda_error() has the code           */
+  TW_ERR_LIMIT = 4,  /* a safety cap was hit (per-utterance: see tw_decode out_status)  */
+  TW_ERR_STATE = 5,  /* call not valid for this handle (e.g. stage needs another mode)  */
+  TW_ERR_TIMEOUT = 6 /* a bounded device-side wait gave up; results are not valid       */
+} tw_status;
+
+enum { TW_MODE_F32 = 0, TW_MODE_BF16 = 1 };
+enum { TW_PRED_STATELESS = 0, TW_PRED_LSTM = 1 };
+
+#define TW_MAX_BEAM 16     /* N <= 16 */
+#define TW_MAX_SEGMENT 64  /* S <= 64 */
+
+/*
+ * The RNN-T pieces the search calls (Sec. 3.1).
+ *   joiner:    z(t,u,.) = W_out . tanh(W_e h_t + W_p g_u) + b_out,  J = softmax(z)
+ *   predictor: stateless  g = emb[last token]         (P == emb_dim; empty prefix -> emb[blank])
+ *              LSTM       lstm_layers stacked cells, gate order (input, forget, cell, output),
+ *                         one bias per layer, g = top layer's h   (P == lstm_hidden);
+ *                         InitPredictor() = one step on the blank token from an all-zero state.
+ * Weight pointers are device float32; in TW_MODE_BF16 the library keeps bf16 copies (exact if the
+ * values are already bf16-representable).  The per-layer pointer tables are HOST arrays of device
+ * pointers.  Nothing passed here is referenced after tw_init returns.
+ */
+typedef struct {
+  int32_t D_enc, P, J, V, blank;
+  int32_t pred_kind, emb_dim, lstm_layers, lstm_hidden;
+  const float* W_e;   /* [J, D_enc] */
+  const float* W_p;   /* [J, P]     */
+  const float* W_out; /* [V, J]     */
+  const float* b_out; /* [V]        */
+  const float* emb;   /* [V, emb_dim] */
+  const float* const* host_lstm_W_ih; /* [lstm_layers] -> [4*Hd, in]  (in = emb_dim, then Hd) */
+  const float* const* host_lstm_W_hh; /* [lstm_layers] -> [4*Hd, Hd] */
+  const float* const* host_lstm_b;    /* [lstm_layers] -> [4*Hd]     */
+} tw_model;
+
+/*
+ * Search parameters (Algorithm 1 inputs N and S) and capacities.
+ *   max_iters_per_segment: safety cap on passes of the inner loop per segment; the paper relies on
+ *     the threshold alone.  When an utterance hits it the rest of its list A is dropped for that
+ *     segment and its status becomes TW_ERR_LIMIT.  0 selects 4*S + 16.
+ *   max_tokens: capacity of a hypothesis' token sequence (U_cap).  An expansion that would exceed
+ *     it is dropped and the utterance's status becomes TW_ERR_LIMIT.  0 selects 512.
+ */
+typedef struct {
+  int32_t N, S, mode;
+  int32_t max_batch, max_T;
+  int32_t max_iters_per_segment;
+  int32_t max_tokens;
+} tw_config;
+
+/* Counters of the last tw_decode (Sec. 4.2: Calls/Frame = calls/frames, Joins/Frame = joins/frames). */
+typedef struct {
+  int64_t frames;        /* sum of utterance lengths                                  */
+  int64_t calls;         /* sum over utterances of inner-loop passes (joiner calls)   */
+  int64_t joins;         /* sum over passes of the frames in that pass' segment       */
+  int64_t steps;         /* batched device steps that did work (one step = one pass for every live utterance) */
+  int64_t rows;          /* sum over steps of live hypothesis rows R                  */
+  int64_t kernel_launches; /* kernels enqueued by the last tw_decode                  */
+  int64_t limit_hits;    /* utterances whose status is TW_ERR_LIMIT                   */
+} tw_stats;
+
+/* Builds a decoder: copies (and in bf16 mode converts) the weights, runs InitPredictor, allocates
+ * the workspace for max_batch utterances of up to max_T frames.  Synchronises the device.
+ * Errors: TW_ERR_ARG for null pointers, N not in [1, TW_MAX_BEAM], S not in [1, TW_MAX_SEGMENT],
+ * V - 1 < N (fewer non-blank tokens than the beam), blank outside [0, V), P inconsistent with the
+ * predictor; TW_ERR_ALLOC / TW_ERR_CUDA otherwise.  *out is NULL on failure. */
+int tw_init(const tw_model* host_model, const tw_config* host_cfg, tw_handle** out);
+int tw_destroy(tw_handle* h);
+
+/*
+ * Algorithm 1 for a batch of B utterances, each decoded independently.
+ *   enc      [B, T, D_enc]  encoder output (computed beforehand, Sec. 3.2); frames at or past
+ *                           lengths[b] are ignored
+ *   lengths  [B]            0 <= lengths[b] <= T (values outside are clamped and flagged TW_ERR_ARG
+ *                           in out_status[b])
+ *   out_tokens [B, N, U_cap] N best token sequences, best first, padded with -1
+ *   out_lens   [B, N]        their lengths; -1 for an unused slot (fewer than N hypotheses)
+ *   out_scores [B, N]        float64 log p, descending; -inf for an unused slot
+ *   out_status [B]           TW_OK, TW_ERR_LIMIT or TW_ERR_ARG per utterance
+ * Every step of the inner loop (joiner over the segment, softmax, Eq. 3-7, AddAndMerge, threshold,
+ * N-best expansions, predictor update) runs on the device; the host only enqueues batches of steps
+ * and polls one completion word between batches.  The call synchronises `stream` before returning.
+ * Returns TW_ERR_LIMIT if any utterance hit a cap (outputs are still valid for the others),
+ * TW_ERR_ARG if B > max_batch, T > max_T or a pointer is null.
+ */
+int tw_decode(tw_handle* h, const float* enc, const int32_t* lengths, int32_t B, int32_t T,
+              int32_t* out_tokens, int32_t* out_lens, double* out_scores, int32_t* out_status,
+              void* stream);
+
+/* Same as tw_decode with HOST buffers: copies the inputs to the device, decodes, copies the four
+ * outputs back.  All copies are on `stream`; synchronises before returning. */
+int tw_decode_host(tw_handle* h, const float* host_enc, const int32_t* host_lengths, int32_t B,
+                   int32_t T, int32_t* host_out_tokens, int32_t* host_out_lens,
+                   double* host_out_scores, int32_t* host_out_status, void* stream);
+
+/* U_cap of this handle (row length of out_tokens). */
+int tw_max_tokens(const tw_handle* h);
+
+/*
+ * Encoder half of the joiner's first layer, E = enc . W_e^T, computed once per frame
+ * (Sec. 3.1 joiner; the split of the first layer is exact algebra).
+ *   enc [rows, D_enc] -> out_E [rows, J]
+ */
+int tw_project_encoder(tw_handle* h, const float* enc, int32_t rows, float* out_E, void* stream);
+
+/*
+ * J = Softmax(Joiner(seg, pred)) of Algorithm 1 for R hypothesis rows, in log space.
+ *   E_seg     [G, S, J]  projected frames of G segments (see tw_project_encoder)
+ *   Pp        [R, J]     projected predictor outputs W_p g of the R rows
+ *   row_group [R]        segment index g of each row, 0 <= g < G
+ *   seg_len   [G]        valid frames of each segment, 1 <= seg_len[g] <= S (NULL: all S)
+ *   out_logp  [R, S, V]  log J(t, r, k); for a frame t >= seg_len the row is the pass-through
+ *                        pattern (0 at blank, -inf elsewhere), which leaves Eq. 3-7 unchanged
+ * Errors: TW_ERR_ARG for null pointers or R, G < 0.  R == 0 is a no-op.
+ */
+int tw_joiner_segment(tw_handle* h, const float* E_seg, const float* Pp, const int32_t* row_group,
+                      const int32_t* seg_len, int32_t G, int32_t R, float* out_logp, void* stream);
+
+/*
+ * Eq. 3-7 for R rows from materialised log-probabilities.
+ *   logp        [R, S, V]  log J
+ *   ld_old      [R, S]     log d_old: log-probability that the row's last token was emitted at
+ *                          frame t (Eq. 2); -inf allowed.  Any common offset per row carries
+ *                          through to the outputs, so callers may pass values relative to the
+ *                          row's score.
+ *   seg_len_row [R]        valid frames per row (NULL: all S)
+ *   out_ldphi   [R]        log delta_phi (Eq. 7)
+ *   out_ldnb    [R, V]     log delta_nb(k) (Eq. 6); -inf at the blank column
+ *   out_la      [R, S]     log a(t) = log sum_{t1<=t} d_old(t1) Bl(t1, t), so that Eq. 5 reads
+ *                          log d(k, t) = out_la[t] + logp[t, k]; -inf for t >= seg_len
+ */
+int tw_expand(tw_handle* h, const float* logp, const float* ld_old, const int32_t* seg_len_row,
+              int32_t R, float* out_ldphi, float* out_ldnb, float* out_la, void* stream);
+
+/*
+ * Joiner, softmax and Eq. 3-7 in one call, without handing log J to the caller (the path tw_decode
+ * takes).  Arguments as in tw_joiner_segment and tw_expand; ld_old is [R, S] and seg_len is per
+ * segment.  R must not exceed max_batch * N.  In TW_MODE_F32 this runs the two stages above through
+ * the handle's own log J buffer.
+ */
+int tw_joiner_expand(tw_handle* h, const float* E_seg, const float* Pp, const int32_t* row_group,
+                     const int32_t* seg_len, const float* ld_old, int32_t G, int32_t R,
+                     float* out_ldphi, float* out_ldnb, float* out_la, void* stream);
+
+/*
+ * UpdatePredictorOutput (Algorithm 1) for R hypotheses at once: one predictor step on `tokens[r]`
+ * from the parent's recurrent state.
+ *   tokens    [R]
+ *   state_in  [R, L, 2, Hd]  per layer h then c (ignored for the stateless predictor; may be NULL)
+ *   state_out [R, L, 2, Hd]  (may be NULL for the stateless predictor)
+ *   out_Pp    [R, J]         W_p g for the joiner
+ * InitPredictor corresponds to tokens = blank with an all-zero state_in.
+ * R must not exceed max_batch * N.
+ */
+int tw_predictor_step(tw_handle* h, const int32_t* tokens, const float* state_in, int32_t R,
+                      float* state_out, float* out_Pp, void* stream);
+
+int tw_get_stats(const tw_handle* h, tw_stats* host_out);
+int tw_last_cuda_error(const tw_handle* h); /* cudaError_t of the last failed CUDA call, 0 if none */
+const char* tw_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TW_H_ */

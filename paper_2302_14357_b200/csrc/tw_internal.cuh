@@ -1,0 +1,128 @@
+// Internal declarations shared by the translation units of libtw.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <math.h>
+
+#include "../../include/tw.h"
+
+namespace tw {
+
+constexpr int kMaxBeam = TW_MAX_BEAM;
+constexpr int kMaxSeg = TW_MAX_SEGMENT;
+constexpr int kMaxLayers = 4;
+
+// ---------------------------------------------------------------------------------------------
+// numerics helpers (accurate libm versions: the fp32 mode must track an fp64 reference to ~1e-6)
+__device__ __forceinline__ float logaddexp_f(float a, float b) {
+  if (a == -INFINITY) return b;
+  if (b == -INFINITY) return a;
+  float m = fmaxf(a, b);
+  return m + log1pf(expf(-fabsf(a - b)));
+}
+__device__ __forceinline__ double logaddexp_d(double a, double b) {
+  if (a == -INFINITY) return b;
+  if (b == -INFINITY) return a;
+  double m = fmax(a, b);
+  return m + log1p(exp(-fabs(a - b)));
+}
+
+// ---------------------------------------------------------------------------------------------
+// SIMT fp32 GEMM  C[m, n] = sum_k A[m, k] * B[n, k] (+ second operand pair) (+ bias[n])
+struct GemmOperand {
+  const float* A;     // rows of length K; row m starts at A + (idx ? idx[m] : m) * ldA
+  const int* idx;     // optional row gather
+  long long ldA;
+  const float* B;     // [N, K] row-major, leading dimension ldB
+  long long ldB;
+  int K;
+};
+
+struct GemmOut {
+  float* C;           // row m written at C + (oidx ? oidx[m] : m) * ldC
+  const int* oidx;
+  long long ldC;
+  const float* bias;  // optional [N]
+};
+
+// M may come from device memory (M_dev != nullptr): CTAs beyond it exit.
+void launch_gemm_f32(const GemmOperand& op1, const GemmOperand& op2, const GemmOut& out,
+                     const int* M_dev, int M_max, int N, cudaStream_t st);
+
+// Joiner rows: hypothesis row r covers frames E[row_e0[r] + t], t < row_slen[r], and the projected
+// predictor output Pp[row_p[r]].
+struct JoinerRows {
+  const float* E;        // [*, J]
+  const int* row_e0;     // [R] first frame row of each hypothesis row
+  const float* Pp;       // [*, J]
+  const int* row_p;      // [R] row into Pp (nullptr: identity)
+  const int* row_slen;   // [R] valid frames (nullptr: S)
+  const int* R_dev;      // device row count (nullptr: use R_max)
+  int R_max, S, J, V;
+};
+// z[(r,t), k] = sum_j tanh(E[e0[r]+t, j] + Pp[p[r], j]) * W_out[k, j] + b_out[k]; rows of padding
+// frames (t >= slen) are left untouched.
+void launch_joiner_f32(const JoinerRows& rows, const float* W_out, const float* b_out, float* z,
+                       cudaStream_t st);
+// in place: z[(r,t), :] -> log softmax; padding frames get (0 at blank, -inf elsewhere)
+void launch_log_softmax(const JoinerRows& rows, int blank, float* z, cudaStream_t st);
+// Eq. 3-7 from materialised log J
+void launch_expand_f32(const float* logp, const float* ld_old, const int* row_slen, const int* R_dev,
+                       int R_max, int S, int V, int blank, float* ldphi, float* ldnb, float* la,
+                       cudaStream_t st);
+// helper for the stage entry points: row_e0[r] = row_group[r] * S, row_slen[r] = seg_len[row_group[r]]
+void launch_rows_from_groups(const int* row_group, const int* seg_len, int R, int S, int* row_e0,
+                             int* row_slen, cudaStream_t st);
+
+// ---------------------------------------------------------------------------------------------
+// Hypothesis state of a batch (structure of arrays in one device workspace).
+enum Scalar { kScR = 0, kScNPred = 1, kScActive = 2, kScSteps = 3, kScCount = 8 };
+
+struct HypState {
+  int B, N, S, V, J, U_cap, I_max, blank;
+  int capB;      // capacity of list B per utterance = N * I_max
+  int capSlot;   // hypothesis slots per utterance = N * (I_max + 1)
+  int L, Hd;     // LSTM layers / hidden (0 for the stateless predictor)
+  int stateless;
+  // per utterance [B]
+  int *len, *t0, *slen, *nA, *nB, *nTop, *iters, *status, *cursor, *n_new, *calls, *joins;
+  // list A: [B][kMaxBeam]
+  int* A_slot; double* A_ls; double* A_ld;   // A_ld [B][kMaxBeam][S]
+  // list B of Algorithm 1 (hypotheses finished for this segment): [B][capB]
+  int* B_slot; double* B_ls; unsigned long long* B_hash; int* B_len;
+  int* B_top;    // [B][kMaxBeam] indices into list B of its best entries, best first
+  int* carry;    // [B][kMaxBeam] slots held by hypotheses carried over from earlier segments
+  // hypothesis slots: [B][capSlot]
+  int* slot_len; unsigned long long* slot_hash; int* slot_tok;  // slot_tok [..][U_cap]
+  float* slot_hc;   // [B*capSlot][L][2][Hd]   (LSTM predictor only)
+  float* slot_Pp;   // [B*capSlot][J]          (LSTM predictor only)
+  // new hypotheses of the current step, per utterance: [B][kMaxBeam] (global slot ids)
+  int *new_slot, *new_par, *new_tok;
+  // compacted rows of the current step: [B*N]
+  int *row_b, *row_e0, *row_p, *row_slen; float* row_ld;   // row_ld [R][S]
+  int *row_off;     // [B]
+  // compacted predictor work list: [B*N]
+  int *pw_new, *pw_par, *pw_tok;
+  int* scalars;           // [kScCount] device scalars
+  long long* rows_total;  // [1]
+  // stage outputs of the current step
+  float *ldphi, *la, *ldnb, *logp;
+  // InitPredictor result (LSTM only): [L][2][Hd], [J]
+  const float* init_hc; const float* init_Pp;
+};
+
+void launch_hyp_init(const HypState& hs, const int* lengths, int B, int T, cudaStream_t st);
+void launch_hyp_step(const HypState& hs, int B, cudaStream_t st);
+void launch_compact(const HypState& hs, int B, int T, cudaStream_t st);
+void launch_finish(const HypState& hs, int B, int* out_tokens, int* out_lens, double* out_scores,
+                   int* out_status, cudaStream_t st);
+
+// LSTM pointwise on slots: gates [n, 4Hd] + parent c -> (h, c) of layer l in the new slot
+void launch_lstm_pointwise_slots(const float* gates, const int* pw_new, const int* pw_par,
+                                 const int* n_dev, int n_max, float* slot_hc, int L, int l, int Hd,
+                                 cudaStream_t st);
+// same on plain [R, L, 2, Hd] state arrays (stage entry point)
+void launch_lstm_pointwise_plain(const float* gates, const float* state_in, float* state_out, int R,
+                                 int L, int l, int Hd, cudaStream_t st);
+
+}  // namespace tw
