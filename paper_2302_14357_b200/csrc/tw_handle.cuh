@@ -1,0 +1,41 @@
+// The decoder handle behind the C ABI.
+#pragma once
+#include <vector>
+
+#include "tw_internal.cuh"
+
+struct tw_handle {
+  // model dimensions and search parameters
+  int D_enc = 0, P = 0, J = 0, V = 0, blank = 0;
+  int pred_kind = 0, emb_dim = 0, L = 0, Hd = 0;
+  int N = 0, S = 0, mode = 0, max_batch = 0, max_T = 0, I_max = 0, U_cap = 0;
+  int R_max = 0;
+
+  // fp32 weights on the device
+  float *W_e = nullptr, *W_p = nullptr, *W_out = nullptr, *b_out = nullptr, *emb = nullptr;
+  float *W_ih[tw::kMaxLayers] = {}, *W_hh[tw::kMaxLayers] = {}, *b_l[tw::kMaxLayers] = {};
+  float* PpTab = nullptr;     // stateless predictor: W_p emb[k] for every token k, [V, J]
+  float* init_hc = nullptr;   // InitPredictor state [L][2][Hd]
+  float* init_Pp = nullptr;   // and its projected output [J]
+
+  tw::HypState hs{};
+  float* E = nullptr;         // projected encoder frames [max_batch * max_T, J]
+  float* gates = nullptr;     // LSTM gate pre-activations [R_max, 4 Hd]
+  int *stage_e0 = nullptr, *stage_slen = nullptr;   // [R_max] scratch of the stage entry points
+
+  // staging of tw_decode_host (allocated on first use)
+  float* st_enc = nullptr; int* st_len = nullptr; int* st_tok = nullptr; int* st_lens = nullptr;
+  double* st_scores = nullptr; int* st_status = nullptr;
+
+  int* host_flag = nullptr;   // pinned copy of the device scalars
+
+  std::vector<void*> dev_allocs;
+  tw_stats stats{};
+  int last_cuda = 0;
+};
+
+namespace tw {
+// stages shared by tw_decode and the stage entry points
+void enqueue_joiner_expand_f32(tw_handle* h, const JoinerRows& rows, const float* ld_old, float* logp,
+                               float* ldphi, float* ldnb, float* la, cudaStream_t st, int* launches);
+}
