@@ -1,0 +1,114 @@
+"""End-to-end parity of tw_decode (fp32 mode) with the oracle's Algorithm 1: identical N-best token
+sequences, log-scores within 1e-4, same Calls/Frame and Joins/Frame counters."""
+import numpy as np
+import pytest
+
+import tw_synth
+from helpers import SCORE_TOL, check_against_oracle, nbest_from_arrays, oracle_model
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(cfg, S, N=None, batch=None, T=None, lengths=None, max_iters=0, mode=0, check=None):
+    from paper_2302_14357_b200.binding import TwDecoder, weights_from_synth
+    N = N or cfg.N
+    m = tw_synth.make_model(cfg)
+    enc, lens = tw_synth.make_encoder_batch(cfg, batch)
+    if T is not None:
+        enc = np.ascontiguousarray(enc[:, :T])
+        lens = np.minimum(lens, T)
+    if lengths is not None:
+        lens = np.asarray(lengths, dtype=np.int32)
+    B = enc.shape[0]
+    dec = TwDecoder(weights_from_synth(m), N=N, S=S, mode=mode, max_batch=B, max_T=enc.shape[1], max_iters_per_segment=max_iters)
+    tokens, olens, scores, status, rc = dec.decode(enc, lens)
+    tokens, olens, scores, status = [x.cpu().numpy() for x in (tokens, olens, scores, status)]
+    stats = dec.stats()
+    om = oracle_model(m)
+    I_max = max_iters or 4 * S + 16
+    calls = joins = 0
+    how = []
+    for b in (range(B) if check is None else check):
+        got = nbest_from_arrays(tokens, olens, scores, b)
+        ok, why, st = check_against_oracle(om, enc[b, :lens[b]], N, S, I_max, got)
+        assert ok, "utterance %d (S=%d): %s" % (b, S, why)
+        assert status[b] == (4 if st.limit_hit else 0)
+        how.append(why)
+        calls += st.calls
+        joins += st.joins
+    if check is None:
+        assert stats["frames"] == int(lens.sum())
+        if all(h == "exact" for h in how):
+            assert stats["calls"] == calls and stats["joins"] == joins
+    assert stats["kernel_launches"] > 0
+    dec.close()
+    return stats, how
+
+
+@pytest.mark.parametrize("S", [1, 2, 3, 7, 40, 64])
+def test_config0_all_segment_sizes(S):
+    _run(tw_synth.get_config("c0"), S)
+
+
+@pytest.mark.parametrize("N", [1, 2, 5, 16])
+def test_config0_beam_sizes(N):
+    _run(tw_synth.get_config("c0"), 3, N=N)
+
+
+def _tiny(pred, layers=1, V=20, seed=5, batch=6, T=23, lo=0):
+    return tw_synth.WorkloadConfig("t", batch, T, (lo, T), 12, pred, 10, layers if pred == "lstm" else 0,
+                                   14 if pred == "lstm" else 0, 16, V, 1.5, 3, (2,), "f32", seed)
+
+
+@pytest.mark.parametrize("pred,layers", [("stateless", 0), ("lstm", 1), ("lstm", 3)])
+@pytest.mark.parametrize("S", [1, 4])
+def test_small_models_ragged_batch(pred, layers, S):
+    """Variable lengths incl. empty and one-frame utterances; S does not divide most lengths."""
+    cfg = _tiny(pred, layers)
+    _run(cfg, S, lengths=[0, 1, 23, 5, 17, 4])
+
+
+def test_iteration_cap_sets_limit_status():
+    cfg = _tiny("stateless", V=12, seed=8).with_(blank_bias=-2.0)
+    stats, _ = _run(cfg, 3, N=3, max_iters=2, lengths=[9, 9, 9, 9, 9, 9])
+    assert stats["limit_hits"] > 0
+
+
+def test_many_merges_small_vocab():
+    """V=3: few distinct sequences, so AddAndMerge fires constantly."""
+    cfg = _tiny("lstm", 1, V=3, seed=12).with_(blank_bias=0.0)
+    _run(cfg, 3, N=2, lengths=[23, 11, 23, 8, 2, 23])
+
+
+@pytest.mark.parametrize("S", [1, 2, 3, 5])
+def test_config1_subset(S):
+    _run(tw_synth.get_config("c1"), S, batch=3, T=90)
+
+
+@pytest.mark.parametrize("S", [3, 10, 50])
+def test_config2_subset(S):
+    _run(tw_synth.get_config("c2"), S, batch=2, T=100)
+
+
+def test_config3_subset():
+    _run(tw_synth.get_config("c3"), 3, batch=2, T=45)
+
+
+def test_config4_shape_subset():
+    _run(tw_synth.get_config("c4"), 10, batch=3, T=40, lengths=[40, 25, 33])
+
+
+def test_decode_host_equals_device_decode():
+    from paper_2302_14357_b200.binding import TwDecoder, weights_from_synth
+    cfg = tw_synth.get_config("c0")
+    m = tw_synth.make_model(cfg)
+    enc, lens = tw_synth.make_encoder_batch(cfg)
+    dec = TwDecoder(weights_from_synth(m), N=2, S=2, max_batch=1, max_T=cfg.T)
+    a = [x.cpu().numpy() for x in dec.decode(enc, lens)[:4]]
+    b = dec.decode_host(enc, lens)[:4]
+    for x, y in zip(a, b):
+        np.testing.assert_array_equal(x, y)
+    # repeated decodes on one handle give the same answer (workspace is re-initialised)
+    c = dec.decode_host(enc, lens)[:4]
+    for x, y in zip(b, c):
+        np.testing.assert_array_equal(x, y)
