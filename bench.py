@@ -1,0 +1,284 @@
+#!/usr/bin/env python
+"""Throughput of the token-wise RNN-T beam search (decoded encoder frames per second).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3] [--segment 3] [--impl ours|reference]
+
+One step = one tw_decode of the whole synthetic batch: every pass of Algorithm 1's inner loop (joiner
+over the segment, softmax, Eq. 3-7, AddAndMerge, threshold, N-best expansions, predictor update) for
+every utterance, plus the once-per-decode encoder projection.  Prints ONE JSON line.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import tw_synth  # noqa: E402
+
+METRIC = "decoded frames/s at N=10,S=3 on 1 B200; joiner+expansion % of roofline"
+UNIT = "frames/s"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c3", choices=sorted(tw_synth.CONFIGS))
+    ap.add_argument("--segment", type=int, default=0, help="segment size S (0: the workload's headline value)")
+    ap.add_argument("--mode", default="auto", choices=["auto", "f32", "bf16"])
+    ap.add_argument("--batch", type=int, default=0, help="utterances per GPU (0: the workload's batch)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-frames", type=int, default=0, help="frames of the CPU-baseline sample (0: auto)")
+    return ap.parse_args()
+
+
+def headline_S(cfg):
+    return 3 if 3 in cfg.S_values else cfg.S_values[0]
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": d["hbm_gbs"], "tflops_burst": d["bf16_tflops"],
+                "tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "tflops_burst": 1590.0, "tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU baseline: the oracle as it stands, on a bounded sample of the same workload
+def oracle_sample(cfg, S, frames, utt=0):
+    from oracle import rnnt_model as rm
+    from oracle import token_wise_search as tws
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    m = tw_synth.make_model(cfg)
+    enc, lens = tw_synth.make_encoder_batch(cfg, batch=utt + 1)
+    om = rm.RnntModel(m.W_e, m.W_p, m.W_out, m.b_out, m.emb, m.lstm_W_ih, m.lstm_W_hh, m.lstm_b)
+    n = int(min(frames, lens[utt]))
+    t0 = time.perf_counter()
+    _, st = tws.token_wise_beam_search(om, enc[utt, :n], cfg.N, S, max_iters=4 * S + 16)
+    dt = time.perf_counter() - t0
+    return {"value": n / dt, "unit": UNIT, "cores": int(cores), "kind": "oracle",
+            "sample": "utterance %d of workload %s, first %d frames, N=%d S=%d, fp64 numpy; %.1f s"
+                      % (utt, cfg.name, n, cfg.N, S, dt),
+            "calls_per_frame": st.calls / max(n, 1), "joins_per_frame": st.joins / max(n, 1)}, dt
+
+
+def auto_cpu_frames(cfg):
+    # sized for roughly 10-30 s of oracle time on a few host cores
+    cost = cfg.J * cfg.V * cfg.N / (640 * 1024 * 10)
+    return int(max(24, min(cfg.T, 400 / max(cost, 0.05))))
+
+
+def run_reference(args, cfg, S):
+    """The reference arm: the fp64 oracle on host cores, each step a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    frames = args.cpu_frames or max(12, auto_cpu_frames(cfg) // 4)
+    for _ in range(args.warmup):
+        oracle_sample(cfg, S, max(4, frames // 4))
+    times, vals, last = [], [], None
+    for k in range(args.steps):
+        last, dt = oracle_sample(cfg, S, frames, utt=0)
+        times.append(dt)
+        vals.append(last["value"])
+    value = frames * len(times) / sum(times) if times else 0.0
+    base = dict(last or {})
+    base["value"] = value
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * sum(times) / max(len(times), 1), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfg.name, "N": cfg.N, "S": S, "sample_frames_per_step": frames},
+            "cpu_baseline": base,
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(device_index), "--query-gpu=" + self.QUERY,
+                                       "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f.read().splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1]))
+                mx.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.f.close()
+        try:
+            os.unlink(self.f.name)
+        except OSError:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def run_ours(args, cfg, S):
+    import torch
+    import torch.distributed as dist
+    from paper_2302_14357_b200.binding import MODE_BF16, MODE_F32, TwDecoder, weights_from_synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the decoder has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    mode_name = "f32" if args.mode == "auto" else args.mode
+    mode = MODE_BF16 if mode_name == "bf16" else MODE_F32
+    B = args.batch or cfg.batch
+    model = tw_synth.make_model(cfg)
+    # every rank decodes its own batch of the same shape (utterances are independent: no exchange)
+    enc_np, len_np = tw_synth.make_encoder_batch(cfg.with_(seed=cfg.seed + 1000 * rank), batch=B)
+    dec = TwDecoder(weights_from_synth(model), N=cfg.N, S=S, mode=mode, max_batch=B, max_T=cfg.T)
+    enc = torch.from_numpy(enc_np).cuda()
+    lens = torch.from_numpy(len_np).cuda()
+    frames = int(len_np.sum())
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        barrier()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record()
+        for _ in range(steps):
+            fn()
+        ev1.record()
+        barrier()
+        ms = ev0.elapsed_time(ev1)
+        if world > 1:
+            t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    for _ in range(args.warmup):
+        dec.decode(enc, lens)
+    # device-resident inputs: the timed region holds only tw_decode calls
+    dec.set_profiling(True)
+    sampler = ClockSampler(local) if rank == 0 else None
+    ms = timed(lambda: dec.decode(enc, lens), args.steps)
+    clocks = sampler.stop() if sampler else None
+    st = dec.stats()            # of the last timed decode (every decode does identical work)
+    dec.set_profiling(False)
+
+    # end to end: pinned host buffers in, host buffers out, copies inside the timed region
+    enc_pin = torch.from_numpy(enc_np).pin_memory()
+    len_pin = torch.from_numpy(len_np).pin_memory()
+    outs = (torch.empty((B, cfg.N, dec.U_cap), dtype=torch.int32).pin_memory().numpy(),
+            torch.empty((B, cfg.N), dtype=torch.int32).pin_memory().numpy(),
+            torch.empty((B, cfg.N), dtype=torch.float64).pin_memory().numpy(),
+            torch.empty((B,), dtype=torch.int32).pin_memory().numpy())
+    e2e_steps = max(1, min(args.steps, 3))
+    dec.decode_host(enc_pin.numpy(), len_pin.numpy(), out=outs)
+    ms_e2e = timed(lambda: dec.decode_host(enc_pin.numpy(), len_pin.numpy(), out=outs), e2e_steps)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    value = world * frames * args.steps / (ms * 1e-3)
+    e2e_value = world * frames * e2e_steps / (ms_e2e * 1e-3)
+    # dominant kernel: the joiner contraction, 2*J*V flops per (row, frame)
+    flops_per_row = 2.0 * cfg.J * cfg.V
+    joiner_s = st["ns_joiner"] * 1e-9
+    achieved = st["joiner_frame_rows"] * flops_per_row / joiner_s / 1e12 if joiner_s > 0 else 0.0
+    peak = peaks["tflops_sustained"]
+    stage_ns = {k: st[k] for k in ("ns_prologue", "ns_predictor", "ns_joiner", "ns_scan", "ns_hyp")}
+    tot_ns = max(1, sum(stage_ns.values()))
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": mode_name, "data": "synthetic",
+        "config": {"workload": cfg.name, "B_per_gpu": B, "T": cfg.T, "N": cfg.N, "S": S, "J": cfg.J, "V": cfg.V,
+                   "mode": mode_name, "l2": "inputs larger than L2 (encoder batch %.0f MB, fresh per-step state)" % (enc_np.nbytes / 1e6),
+                   "parallelism": "independent utterance batches per GPU, no collective"},
+        "calls_per_frame": st["calls"] / max(st["frames"], 1), "joins_per_frame": st["joins"] / max(st["frames"], 1),
+        "device_steps_per_decode": st["steps"], "avg_rows_per_step": st["rows"] / max(st["steps"], 1),
+        "limit_hits": st["limit_hits"],
+        "stage_share": {k[3:]: round(v / tot_ns, 4) for k, v in stage_ns.items()},
+        "stage_ms_per_decode": {k[3:]: round(v * 1e-6, 3) for k, v in stage_ns.items()},
+        "roofline": {"kernel": "joiner contraction tanh(E+Pp).W_out^T", "bound": "tensor", "achieved": achieved, "peak": peak,
+                     "unit": "TFLOP/s", "frac": achieved / peak if peak else None, "traffic": None,
+                     "peak_source": "%s bf16 sustained" % peaks["source"],
+                     "avg_launch_us": 1e6 * joiner_s / max(st["joiner_launches"], 1),
+                     "flops_per_launch": st["joiner_frame_rows"] * flops_per_row / max(st["joiner_launches"], 1)},
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(enc_np.nbytes + len_np.nbytes),
+                "d2h_bytes_per_step": int(sum(o.nbytes for o in outs))},
+        "gpu_launches": int(st["kernel_launches"] * args.steps),
+        "clocks": clocks,
+    }
+    if not args.no_cpu_baseline and world == 1:
+        line["cpu_baseline"], _ = oracle_sample(cfg, S, args.cpu_frames or auto_cpu_frames(cfg))
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    cfg = tw_synth.get_config(args.workload)
+    S = args.segment or headline_S(cfg)
+    if args.impl == "reference":
+        run_reference(args, cfg, S)
+    else:
+        run_ours(args, cfg, S)
+
+
+if __name__ == "__main__":
+    main()

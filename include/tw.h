@@ -96,6 +96,14 @@ typedef struct {
   int64_t rows;          /* sum over steps of live hypothesis rows R                  */
   int64_t kernel_launches; /* kernels enqueued by the last tw_decode                  */
   int64_t limit_hits;    /* utterances whose status is TW_ERR_LIMIT                   */
+  int64_t joiner_frame_rows; /* sum over steps of (rows x frames of their segment) = joiner GEMM rows M */
+  /* device time per stage in nanoseconds, summed over the decode; zero unless tw_set_profiling(h, 1) */
+  int64_t ns_prologue;   /* E = enc W_e^T and list initialisation                      */
+  int64_t ns_predictor;  /* UpdatePredictorOutput                                      */
+  int64_t ns_joiner;     /* joiner contraction (+ softmax and Eq. 3-7 where fused)     */
+  int64_t ns_scan;       /* softmax and Eq. 3-7 where they are separate kernels        */
+  int64_t ns_hyp;        /* AddAndMerge, threshold, N-best expansions, compaction      */
+  int64_t joiner_launches; /* launches summed in ns_joiner                             */
 } tw_stats;
 
 /* Builds a decoder: copies (and in bf16 mode converts) the weights, runs InitPredictor, allocates
@@ -194,6 +202,9 @@ int tw_joiner_expand(tw_handle* h, const float* E_seg, const float* Pp, const in
 int tw_predictor_step(tw_handle* h, const int32_t* tokens, const float* state_in, int32_t R,
                       float* state_out, float* out_Pp, void* stream);
 
+/* Per-stage device timing of tw_decode with CUDA events on the decode stream (adds two event records
+ * per stage per step); off by default. */
+int tw_set_profiling(tw_handle* h, int on);
 int tw_get_stats(const tw_handle* h, tw_stats* host_out);
 int tw_last_cuda_error(const tw_handle* h); /* cudaError_t of the last failed CUDA call, 0 if none */
 const char* tw_strerror(int status);

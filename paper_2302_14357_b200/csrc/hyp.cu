@@ -103,7 +103,7 @@ __device__ __forceinline__ bool better(float v, int k, float v2, int k2) {
 
 __global__ void __launch_bounds__(kThreads) hyp_step_kernel(HypState hs) {
   __shared__ int s_scratch[kThreads / 32];
-  __shared__ int s_nB, s_hasthr, s_found, s_nkeep, s_ntot;
+  __shared__ int s_nB, s_hasthr, s_nkeep, s_ntot;
   __shared__ int s_touched[kMaxBeam];
   __shared__ double s_Als[kMaxBeam];
   __shared__ int s_Aslot[kMaxBeam];
@@ -161,7 +161,7 @@ __global__ void __launch_bounds__(kThreads) hyp_step_kernel(HypState hs) {
       start = cand + 1;
     }
     if (tid == 0) {
-      const double val = s_Als[h] + (double)hs.ldphi[r0 + h];
+      const double val = s_Als[h] + (hs.ldphi_d ? hs.ldphi_d[r0 + h] : (double)hs.ldphi[r0 + h]);
       if (found >= 0) {
         hs.B_ls[bB + found] = logaddexp_d(hs.B_ls[bB + found], val);
         s_touched[h] = found;
@@ -331,7 +331,8 @@ __global__ void __launch_bounds__(kThreads) hyp_step_kernel(HypState hs) {
       double v = -INFINITY;
       if (tid < slen && hs.logp != nullptr) {
         const long long r = r0 + h;
-        v = s_Als[h] + (double)hs.la[r * S + tid] + (double)hs.logp[(r * S + tid) * V + k];
+        const double a = hs.la_d ? hs.la_d[r * S + tid] : (double)hs.la[r * S + tid];
+        v = s_Als[h] + a + (double)hs.logp[(r * S + tid) * V + k];
       }
       s_newld[i][tid] = v;
     }
@@ -356,9 +357,9 @@ __global__ void __launch_bounds__(kThreads) hyp_step_kernel(HypState hs) {
 // into the predictor's work list.
 __global__ void __launch_bounds__(1024) compact_kernel(HypState hs, int B, int T) {
   __shared__ int s_a[1024], s_n[1024];
-  __shared__ int s_base_a, s_base_n;
+  __shared__ int s_base_a, s_base_n, s_frames;
   const int tid = threadIdx.x;
-  if (tid == 0) { s_base_a = 0; s_base_n = 0; }
+  if (tid == 0) { s_base_a = 0; s_base_n = 0; s_frames = 0; }
   __syncthreads();
   for (int b0 = 0; b0 < B; b0 += 1024) {
     const int b = b0 + tid;
@@ -378,6 +379,7 @@ __global__ void __launch_bounds__(1024) compact_kernel(HypState hs, int B, int T
     if (b < B) {
       hs.row_off[b] = off_a;
       const int t0 = hs.t0[b], sl = hs.slen[b];
+      if (a > 0) atomicAdd(&s_frames, a * sl);
       for (int h = 0; h < a; ++h) {
         const int r = off_a + h;
         const int slot = hs.A_slot[b * kMaxBeam + h];
@@ -413,7 +415,7 @@ __global__ void __launch_bounds__(1024) compact_kernel(HypState hs, int B, int T
     hs.scalars[kScR] = R;
     hs.scalars[kScNPred] = s_base_n;
     hs.scalars[kScActive] = R > 0;
-    if (R > 0) { hs.scalars[kScSteps] += 1; *hs.rows_total += R; }
+    if (R > 0) { hs.scalars[kScSteps] += 1; hs.rows_total[0] += R; hs.rows_total[1] += s_frames; }
   }
 }
 

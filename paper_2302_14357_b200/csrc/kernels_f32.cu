@@ -193,7 +193,8 @@ __global__ void __launch_bounds__(256) expand_f32_kernel(const float* __restrict
                                                          const float* __restrict__ ld_old,
                                                          const int* row_slen, const int* R_dev,
                                                          int R_max, int S, int V, int blank,
-                                                         float* ldphi, float* ldnb, float* la_out) {
+                                                         float* ldphi, float* ldnb, float* la_out,
+                                                         double* ldphi_d, double* la_d) {
   __shared__ float la[kMaxSeg];
   const int R = R_dev ? *R_dev : R_max;
   const int r = blockIdx.x;
@@ -201,16 +202,22 @@ __global__ void __launch_bounds__(256) expand_f32_kernel(const float* __restrict
   const int sl = row_slen ? row_slen[r] : S;
   const float* lp = logp + (long long)r * S * V;
   if (threadIdx.x == 0) {
-    float a = ld_old[(long long)r * S];
+    // the recursion is S steps long and its values grow to hundreds of nats: carry it in float64
+    double a = (double)ld_old[(long long)r * S];
+    double phi = -INFINITY;
     for (int t = 0; t < sl; ++t) {
-      la[t] = a;
-      float lb = lp[(long long)t * V + blank];
-      float nxt = a + lb;                       // -inf + finite stays -inf
-      if (t + 1 < sl) a = logaddexp_f(nxt, ld_old[(long long)r * S + t + 1]);
-      else ldphi[r] = nxt;
+      la[t] = (float)a;
+      if (la_d) la_d[(long long)r * S + t] = a;
+      const double nxt = a + (double)lp[(long long)t * V + blank];   // -inf + finite stays -inf
+      if (t + 1 < sl) a = logaddexp_d(nxt, (double)ld_old[(long long)r * S + t + 1]);
+      else phi = nxt;
     }
-    for (int t = (sl > 0 ? sl : 0); t < S; ++t) la[t] = -INFINITY;
-    if (sl <= 0) ldphi[r] = -INFINITY;
+    for (int t = (sl > 0 ? sl : 0); t < S; ++t) {
+      la[t] = -INFINITY;
+      if (la_d) la_d[(long long)r * S + t] = -INFINITY;
+    }
+    ldphi[r] = (float)phi;
+    if (ldphi_d) ldphi_d[r] = phi;
   }
   __syncthreads();
   if (threadIdx.x < S) la_out[(long long)r * S + threadIdx.x] = la[threadIdx.x];
@@ -267,10 +274,10 @@ void launch_log_softmax(const JoinerRows& rows, int blank, float* z, cudaStream_
 
 void launch_expand_f32(const float* logp, const float* ld_old, const int* row_slen, const int* R_dev,
                        int R_max, int S, int V, int blank, float* ldphi, float* ldnb, float* la,
-                       cudaStream_t st) {
+                       double* ldphi_d, double* la_d, cudaStream_t st) {
   if (R_max <= 0) return;
   expand_f32_kernel<<<R_max, 256, 0, st>>>(logp, ld_old, row_slen, R_dev, R_max, S, V, blank, ldphi,
-                                           ldnb, la);
+                                           ldnb, la, ldphi_d, la_d);
 }
 
 void launch_rows_from_groups(const int* row_group, const int* seg_len, int R, int S, int* row_e0,

@@ -128,15 +128,17 @@ int build_workspace(tw_handle* h) {
   for (int** p : per_row) TW_TRY(dev_alloc(h, p, R));
   TW_TRY(dev_alloc(h, &hs.row_ld, R * S));
   TW_TRY(dev_alloc(h, &hs.scalars, (size_t)kScCount));
-  TW_TRY(dev_alloc(h, &hs.rows_total, (size_t)1));
+  TW_TRY(dev_alloc(h, &hs.rows_total, (size_t)2));
   TW_TRY(dev_alloc(h, &hs.ldphi, R));
   TW_TRY(dev_alloc(h, &hs.la, R * S));
+  TW_TRY(dev_alloc(h, &hs.ldphi_d, R));
+  TW_TRY(dev_alloc(h, &hs.la_d, R * S));
   TW_TRY(dev_alloc(h, &hs.ldnb, R * h->V));
   TW_TRY(dev_alloc(h, &hs.logp, R * S * h->V));
   TW_TRY(dev_alloc(h, &h->E, nb * h->max_T * h->J));
   TW_CUDA(h, cudaMemset(hs.scalars, 0, kScCount * sizeof(int)));
-  TW_CUDA(h, cudaMemset(hs.rows_total, 0, sizeof(long long)));
-  TW_CUDA(h, cudaHostAlloc((void**)&h->host_flag, (kScCount + 2) * sizeof(long long), cudaHostAllocDefault));
+  TW_CUDA(h, cudaMemset(hs.rows_total, 0, 2 * sizeof(long long)));
+  TW_CUDA(h, cudaHostAlloc((void**)&h->host_flag, (kScCount + 4) * sizeof(long long), cudaHostAllocDefault));
   return TW_OK;
 }
 
@@ -193,11 +195,12 @@ int init_impl(tw_handle* h, const tw_model* m, const tw_config* c) {
 
 namespace tw {
 void enqueue_joiner_expand_f32(tw_handle* h, const JoinerRows& rows, const float* ld_old, float* logp,
-                               float* ldphi, float* ldnb, float* la, cudaStream_t st, int* launches) {
+                               float* ldphi, float* ldnb, float* la, double* ldphi_d, double* la_d,
+                               cudaStream_t st, int* launches) {
   launch_joiner_f32(rows, h->W_out, h->b_out, logp, st);
   launch_log_softmax(rows, h->blank, logp, st);
   launch_expand_f32(logp, ld_old, rows.row_slen, rows.R_dev, rows.R_max, rows.S, rows.V, h->blank, ldphi,
-                    ldnb, la, st);
+                    ldnb, la, ldphi_d, la_d, st);
   *launches += 3;
 }
 }  // namespace tw
@@ -239,6 +242,7 @@ int tw_destroy(tw_handle* h) {
   if (!h) return TW_ERR_ARG;
   cudaDeviceSynchronize();
   for (void* p : h->dev_allocs) cudaFree(p);
+  for (cudaEvent_t e : h->events) cudaEventDestroy(e);
   if (h->host_flag) cudaFreeHost(h->host_flag);
   delete h;
   return TW_OK;
@@ -246,6 +250,12 @@ int tw_destroy(tw_handle* h) {
 
 int tw_max_tokens(const tw_handle* h) { return h ? h->U_cap : -1; }
 int tw_last_cuda_error(const tw_handle* h) { return h ? h->last_cuda : 0; }
+
+int tw_set_profiling(tw_handle* h, int on) {
+  if (!h) return TW_ERR_ARG;
+  h->profiling = on != 0;
+  return TW_OK;
+}
 
 int tw_get_stats(const tw_handle* h, tw_stats* out) {
   if (!h || !out) return TW_ERR_ARG;

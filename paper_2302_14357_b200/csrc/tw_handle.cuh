@@ -29,6 +29,11 @@ struct tw_handle {
 
   int* host_flag = nullptr;   // pinned copy of the device scalars
 
+  // optional per-stage timing of tw_decode (tw_set_profiling): pooled events and the stage each closes
+  bool profiling = false;
+  std::vector<cudaEvent_t> events;
+  std::vector<int> marks;
+
   std::vector<void*> dev_allocs;
   tw_stats stats{};
   int last_cuda = 0;
@@ -37,5 +42,6 @@ struct tw_handle {
 namespace tw {
 // stages shared by tw_decode and the stage entry points
 void enqueue_joiner_expand_f32(tw_handle* h, const JoinerRows& rows, const float* ld_old, float* logp,
-                               float* ldphi, float* ldnb, float* la, cudaStream_t st, int* launches);
+                               float* ldphi, float* ldnb, float* la, double* ldphi_d, double* la_d,
+                               cudaStream_t st, int* launches);
 }

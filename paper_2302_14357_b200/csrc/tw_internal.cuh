@@ -69,7 +69,7 @@ void launch_log_softmax(const JoinerRows& rows, int blank, float* z, cudaStream_
 // Eq. 3-7 from materialised log J
 void launch_expand_f32(const float* logp, const float* ld_old, const int* row_slen, const int* R_dev,
                        int R_max, int S, int V, int blank, float* ldphi, float* ldnb, float* la,
-                       cudaStream_t st);
+                       double* ldphi_d, double* la_d, cudaStream_t st);   // float64 copies optional
 // helper for the stage entry points: row_e0[r] = row_group[r] * S, row_slen[r] = seg_len[row_group[r]]
 void launch_rows_from_groups(const int* row_group, const int* seg_len, int R, int S, int* row_e0,
                              int* row_slen, cudaStream_t st);
@@ -104,9 +104,10 @@ struct HypState {
   // compacted predictor work list: [B*N]
   int *pw_new, *pw_par, *pw_tok;
   int* scalars;           // [kScCount] device scalars
-  long long* rows_total;  // [1]
+  long long* rows_total;  // [2]: sum over steps of rows R, and of rows x their segment's frames
   // stage outputs of the current step
   float *ldphi, *la, *ldnb, *logp;
+  double *ldphi_d, *la_d;   // float64 copies of ldphi / la (nullptr: use the float32 ones)
   // InitPredictor result (LSTM only): [L][2][Hd], [J]
   const float* init_hc; const float* init_Pp;
 };

@@ -30,7 +30,8 @@ def _allclose_inf(a, b, tol):
     inf_a, inf_b = np.isneginf(a), np.isneginf(b)
     assert np.array_equal(inf_a, inf_b)
     assert np.all(np.isfinite(a[~inf_a]))
-    np.testing.assert_allclose(a[~inf_a], b[~inf_a], rtol=0, atol=tol)
+    # outputs are float32: beyond the stage tolerance allow the rounding of the stored value itself
+    np.testing.assert_allclose(a[~inf_a], b[~inf_a], rtol=1.2e-7, atol=tol)
 
 
 @pytest.mark.parametrize("S,seg_lens", [(1, None), (3, None), (5, [5, 2, 4]), (17, [17, 1, 9])])
