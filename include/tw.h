@@ -202,6 +202,37 @@ int tw_joiner_expand(tw_handle* h, const float* E_seg, const float* Pp, const in
 int tw_predictor_step(tw_handle* h, const int32_t* tokens, const float* state_in, int32_t R,
                       float* state_out, float* out_Pp, void* stream);
 
+/*
+ * Joiner, softmax and Eq. 3-7 for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a packaging of tw_joiner_expand, not another operation.)
+ *
+ * Who needs it: a process whose GPU memory already belongs to someone else's allocator, for instance
+ * an inference server that reserved all of HBM for its own pool at start-up, or a latency-critical
+ * loop in which a cudaMalloc / cudaFree would stall every stream of the device.  Such a caller cannot
+ * afford tw_init, which allocates a workspace.  This call takes no handle: the caller passes the two
+ * joiner weights it needs as ordinary inputs, and the intermediate log J tensor is kept in a fixed
+ * array inside the library image (about 16 MiB per GPU that loads the library, held until the
+ * process exits).  The call itself never calls cudaMalloc, cudaFree or any allocating routine.
+ *
+ *   W_out [V, J], b_out [V]   joiner output layer (float32, device)
+ *   the remaining arguments are those of tw_joiner_expand, computed in float32
+ * Limits: R <= TW_NOALLOC_MAX_ROWS and R * S * V <= TW_NOALLOC_MAX_ELEMS; a larger request returns
+ * TW_ERR_LIMIT and enqueues nothing.  Other bad arguments return TW_ERR_ARG.
+ * The first call on each device looks up the device address of the fixed array (with that device
+ * current); make that first call outside any stream capture.
+ * All calls on a device share the one array, which keeps whatever the previous call left in it.
+ * Nothing in it has to start at zero: each call overwrites every element it later reads.  Two calls
+ * that overlap on the GPU (different streams, or different host threads) race on the array and give
+ * wrong results; serialise them.
+ */
+#define TW_NOALLOC_MAX_ROWS 4096
+#define TW_NOALLOC_MAX_ELEMS (4 * 1024 * 1024)
+int tw_joiner_expand_noalloc(const float* W_out, const float* b_out, int32_t J, int32_t V, int32_t S,
+                             int32_t blank, const float* E_seg, const float* Pp,
+                             const int32_t* row_group, const int32_t* seg_len, const float* ld_old,
+                             int32_t G, int32_t R, float* out_ldphi, float* out_ldnb, float* out_la,
+                             void* stream);
+
 /* Per-stage device timing of tw_decode with CUDA events on the decode stream (adds two event records
  * per stage per step); off by default. */
 int tw_set_profiling(tw_handle* h, int on);

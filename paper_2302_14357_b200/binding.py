@@ -12,6 +12,7 @@ TW_OK, TW_ERR_ARG, TW_ERR_ALLOC, TW_ERR_CUDA, TW_ERR_LIMIT, TW_ERR_STATE, TW_ERR
 EXPORTED_SYMBOLS = [
     "tw_init", "tw_destroy", "tw_decode", "tw_decode_host", "tw_max_tokens", "tw_project_encoder",
     "tw_joiner_segment", "tw_expand", "tw_joiner_expand", "tw_predictor_step", "tw_get_stats", "tw_set_profiling",
+    "tw_joiner_expand_noalloc",
     "tw_last_cuda_error", "tw_strerror",
 ]
 
@@ -67,6 +68,7 @@ def load_library() -> C.CDLL:
     lib.tw_predictor_step.argtypes = [vp, vp, vp, i32, vp, vp, vp]
     lib.tw_get_stats.argtypes = [vp, C.POINTER(_Stats)]
     lib.tw_set_profiling.argtypes = [vp, C.c_int]
+    lib.tw_joiner_expand_noalloc.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp]
     lib.tw_last_cuda_error.argtypes = [vp]
     lib.tw_strerror.argtypes = [C.c_int]
     lib.tw_strerror.restype = C.c_char_p
@@ -252,3 +254,26 @@ def weights_from_synth(m) -> Dict:
     """tw_model fields from a tw_synth.SyntheticModel (plain attribute access, no arithmetic)."""
     return dict(W_e=m.W_e, W_p=m.W_p, W_out=m.W_out, b_out=m.b_out, emb=m.emb,
                 lstm_W_ih=list(m.lstm_W_ih), lstm_W_hh=list(m.lstm_W_hh), lstm_b=list(m.lstm_b))
+
+
+NOALLOC_MAX_ROWS = 4096
+NOALLOC_MAX_ELEMS = 4 * 1024 * 1024
+
+
+def joiner_expand_noalloc(W_out, b_out, S, blank, E_seg, Pp, row_group, seg_len, ld_old):
+    """tw_joiner_expand_noalloc: joiner + softmax + Eq. 3-7 without a handle and without any device
+    allocation inside the library (its scratch is a fixed array in the library image).  All arguments
+    are CUDA tensors the caller already owns (float32, int32 for row_group / seg_len); the three
+    outputs are allocated here, by the caller's side, before the call.  Returns (status, ldphi, ldnb, la)."""
+    import torch
+    lib = load_library()
+    V, J = W_out.shape
+    G, R = E_seg.shape[0], Pp.shape[0]
+    dev = W_out.device
+    ldphi = torch.empty((R,), dtype=torch.float32, device=dev)
+    ldnb = torch.empty((R, V), dtype=torch.float32, device=dev)
+    la = torch.empty((R, S), dtype=torch.float32, device=dev)
+    st = lib.tw_joiner_expand_noalloc(W_out.data_ptr(), b_out.data_ptr(), J, V, S, blank, E_seg.data_ptr(), Pp.data_ptr(),
+                                      row_group.data_ptr(), _ptr(seg_len), ld_old.data_ptr(), G, R, ldphi.data_ptr(),
+                                      ldnb.data_ptr(), la.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    return st, ldphi, ldnb, la
