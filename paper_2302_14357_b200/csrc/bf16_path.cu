@@ -1,0 +1,77 @@
+// Elementwise kernels of the bf16 path: conversions, operand gathers and the joiner's A operand.
+#include "bf16_path.cuh"
+
+namespace tw {
+
+namespace {
+
+__global__ void f32_to_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, long long n) {
+  long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  if (i + 3 < n && ((reinterpret_cast<uintptr_t>(src + i) & 15) == 0)) {
+    const float4 v = *reinterpret_cast<const float4*>(src + i);
+    __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
+    *reinterpret_cast<__nv_bfloat162*>(dst + i) = a;
+    *reinterpret_cast<__nv_bfloat162*>(dst + i + 2) = b;
+  } else {
+    for (int j = 0; j < 4 && i + j < n; ++j) dst[i + j] = __float2bfloat16_rn(src[i + j]);
+  }
+}
+
+__global__ void gather_concat_bf16_kernel(const float* __restrict__ src1, const int* idx1, long long ld1, int K1,
+                                          const float* __restrict__ src2, const int* idx2, long long ld2, int K2,
+                                          const int* n_dev, int n_max, __nv_bfloat16* __restrict__ dst) {
+  const int n = n_dev ? *n_dev : n_max;
+  const int r = blockIdx.x;
+  if (r >= n) return;
+  const int K = K1 + K2;
+  const float* a = src1 + (long long)(idx1 ? idx1[r] : r) * ld1;
+  const float* b = K2 > 0 ? src2 + (long long)(idx2 ? idx2[r] : r) * ld2 : nullptr;
+  __nv_bfloat16* d = dst + (long long)r * K;
+  for (int k = threadIdx.x; k < K; k += blockDim.x) d[k] = __float2bfloat16_rn(k < K1 ? a[k] : b[k - K1]);
+}
+
+__device__ __forceinline__ float tanh_fast(float x) {
+  float y;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// one CTA per (row, frame); the tanh error of the approximate instruction (about 2^-11) is below the
+// bf16 rounding (2^-9) of the stored operand
+__global__ void joiner_A_bf16_kernel(JoinerRows jr, __nv_bfloat16* __restrict__ A) {
+  const int R = jr.R_dev ? *jr.R_dev : jr.R_max;
+  const int m = blockIdx.x;
+  const int r = m / jr.S, t = m - r * jr.S;
+  if (r >= R) return;
+  const int sl = jr.row_slen ? jr.row_slen[r] : jr.S;
+  __nv_bfloat16* dst = A + (long long)m * jr.J;
+  if (t >= sl) {
+    for (int j = threadIdx.x; j < jr.J; j += blockDim.x) dst[j] = __float2bfloat16_rn(0.f);
+    return;
+  }
+  const float* e = jr.E + (long long)(jr.row_e0[r] + t) * jr.J;
+  const float* p = jr.Pp + (long long)(jr.row_p ? jr.row_p[r] : r) * jr.J;
+  for (int j = threadIdx.x; j < jr.J; j += blockDim.x) dst[j] = __float2bfloat16_rn(tanh_fast(e[j] + p[j]));
+}
+
+}  // namespace
+
+void launch_f32_to_bf16(const float* src, __nv_bfloat16* dst, long long n, cudaStream_t st) {
+  if (n <= 0) return;
+  const long long threads = (n + 3) / 4;
+  f32_to_bf16_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(src, dst, n);
+}
+
+void launch_gather_concat_bf16(const float* src1, const int* idx1, long long ld1, int K1, const float* src2,
+                               const int* idx2, long long ld2, int K2, const int* n_dev, int n_max,
+                               __nv_bfloat16* dst, cudaStream_t st) {
+  if (n_max <= 0) return;
+  gather_concat_bf16_kernel<<<n_max, 256, 0, st>>>(src1, idx1, ld1, K1, src2, idx2, ld2, K2, n_dev, n_max, dst);
+}
+
+void launch_joiner_A_bf16(const JoinerRows& rows, __nv_bfloat16* A, cudaStream_t st) {
+  if (rows.R_max <= 0) return;
+  joiner_A_bf16_kernel<<<rows.R_max * rows.S, 256, 0, st>>>(rows, A);
+}
+
+}  // namespace tw

@@ -1,0 +1,45 @@
+// TW_MODE_BF16: bf16 operands on the tcgen05 tensor cores, fp32 accumulation and fp32 epilogues.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "tw_internal.cuh"
+
+namespace tw {
+
+struct GemmBf16Params {
+  const int* M_dev;   // device row count (nullptr: use M); CTAs beyond it exit
+  int M, N, K;        // M is the maximum when M_dev is given
+  float* C;           // row m written at C + (oidx ? oidx[m] : m) * ldC
+  const int* oidx;
+  long long ldC;
+  const float* bias;  // optional [N]
+  int* err;           // device error word, raised by a wait that gave up
+};
+
+// 2-D bf16 tensor map over a row-major [rows, K] matrix, box = 64 x box_rows, 128-byte swizzle.
+// Requires K % 8 == 0 and a 16-byte aligned base.
+int make_tmap_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint64_t K, uint32_t box_rows);
+int gemm_bf16_setup();
+// tmB128 / tmB256: maps of the same B matrix with 128- and 256-row boxes
+void launch_gemm_bf16(const CUtensorMap& tmA, const CUtensorMap& tmB128, const CUtensorMap& tmB256,
+                      const GemmBf16Params& p, cudaStream_t st);
+
+// A bf16 matrix with its tensor maps
+struct Bf16Mat {
+  __nv_bfloat16* ptr = nullptr;
+  long long rows = 0, K = 0;
+  CUtensorMap as_A;            // box 128 rows
+  CUtensorMap as_B128, as_B256;
+};
+
+// elementwise helpers ---------------------------------------------------------------------------
+void launch_f32_to_bf16(const float* src, __nv_bfloat16* dst, long long n, cudaStream_t st);
+// dst[r, 0:K1] = src1 row (idx1 ? idx1[r] : r), dst[r, K1:K1+K2] = src2 row (idx2 ? idx2[r] : r)
+void launch_gather_concat_bf16(const float* src1, const int* idx1, long long ld1, int K1, const float* src2,
+                               const int* idx2, long long ld2, int K2, const int* n_dev, int n_max,
+                               __nv_bfloat16* dst, cudaStream_t st);
+// joiner A operand: A[(r, t), j] = tanh(E[e0[r]+t, j] + Pp[p[r], j]) as bf16; zero rows for padding frames
+void launch_joiner_A_bf16(const JoinerRows& rows, __nv_bfloat16* A, cudaStream_t st);
+
+}  // namespace tw

@@ -413,6 +413,7 @@ __global__ void __launch_bounds__(1024) compact_kernel(HypState hs, int B, int T
   if (tid == 0) {
     const int R = s_base_a;
     hs.scalars[kScR] = R;
+    hs.scalars[kScM] = R * hs.S;
     hs.scalars[kScNPred] = s_base_n;
     hs.scalars[kScActive] = R > 0;
     if (R > 0) { hs.scalars[kScSteps] += 1; hs.rows_total[0] += R; hs.rows_total[1] += s_frames; }
@@ -478,20 +479,12 @@ void launch_finish(const HypState& hs, int B, int* out_tokens, int* out_lens, do
                    int* out_status, cudaStream_t st) {
   if (B > 0) finish_kernel<<<B, kThreads, 0, st>>>(hs, out_tokens, out_lens, out_scores, out_status);
 }
-void launch_lstm_pointwise_slots(const float* gates, const int* pw_new, const int* pw_par,
-                                 const int* n_dev, int n_max, float* slot_hc, int L, int l, int Hd,
-                                 cudaStream_t st) {
+void launch_lstm_pointwise(const float* gates, const int* idx_out, const int* idx_in, const int* n_dev,
+                           int n_max, const float* hc_in, float* hc_out, int L, int l, int Hd, cudaStream_t st) {
   if (n_max <= 0) return;
   const long long tot = (long long)n_max * Hd;
-  lstm_pointwise_kernel<<<(unsigned)((tot + 255) / 256), 256, 0, st>>>(gates, pw_new, pw_par, n_dev, n_max,
-                                                                      slot_hc, slot_hc, L, l, Hd);
-}
-void launch_lstm_pointwise_plain(const float* gates, const float* state_in, float* state_out, int R,
-                                 int L, int l, int Hd, cudaStream_t st) {
-  if (R <= 0) return;
-  const long long tot = (long long)R * Hd;
-  lstm_pointwise_kernel<<<(unsigned)((tot + 255) / 256), 256, 0, st>>>(gates, nullptr, nullptr, nullptr, R,
-                                                                      state_in, state_out, L, l, Hd);
+  lstm_pointwise_kernel<<<(unsigned)((tot + 255) / 256), 256, 0, st>>>(gates, idx_out, idx_in, n_dev, n_max, hc_in,
+                                                                      hc_out, L, l, Hd);
 }
 
 }  // namespace tw

@@ -37,33 +37,78 @@ int copy_weight(tw_handle* h, float** dst, const float* src, size_t count) {
   return TW_OK;
 }
 
-// One predictor step on plain arrays (see tw_predictor_step).
-int enqueue_predictor_plain(tw_handle* h, const int* tokens, const float* state_in, int R,
-                            float* state_out, float* out_Pp, cudaStream_t st, int* launches) {
+// fp32 -> bf16 copy of a [rows, K] matrix with its tensor maps
+int make_bf16_mat(tw_handle* h, Bf16Mat* m, const float* src, long long rows, long long K, bool as_A, bool as_B) {
+  m->rows = rows; m->K = K;
+  TW_TRY(dev_alloc(h, &m->ptr, (size_t)(rows * K)));
+  if (src) launch_f32_to_bf16(src, m->ptr, rows * K, 0);
+  else TW_CUDA(h, cudaMemset(m->ptr, 0, (size_t)(rows * K) * sizeof(__nv_bfloat16)));
+  if (as_A) TW_TRY(make_tmap_bf16(&m->as_A, m->ptr, rows, K, 128));
+  if (as_B) {
+    TW_TRY(make_tmap_bf16(&m->as_B128, m->ptr, rows, K, 128));
+    TW_TRY(make_tmap_bf16(&m->as_B256, m->ptr, rows, K, 256));
+  }
+  return TW_OK;
+}
+
+void gemm_bf16(tw_handle* h, const Bf16Mat& A, const Bf16Mat& B, const int* M_dev, int M, float* C, const int* oidx,
+               long long ldC, const float* bias, cudaStream_t st) {
+  GemmBf16Params p{M_dev, M, (int)B.rows, (int)A.K, C, oidx, ldC, bias, h->bf.err};
+  launch_gemm_bf16(A.as_A, B.as_B128, B.as_B256, p, st);
+}
+
+// UpdatePredictorOutput for n hypotheses: one predictor step on tok[i] from the state at row
+// (idx_in ? idx_in[i] : i) of hc_in, written to row (idx_out ? idx_out[i] : i) of hc_out; the projected
+// output W_p g goes to row (idx_out ? idx_out[i] : i) of Pp_out.  State rows are [L][2][Hd].
+void enqueue_predictor(tw_handle* h, const int* tok, const float* hc_in, const int* idx_in, float* hc_out,
+                       const int* idx_out, float* Pp_out, const int* n_dev, int n_max, cudaStream_t st,
+                       int* launches) {
+  GemmOperand none{};
   if (h->pred_kind == TW_PRED_STATELESS) {
-    GemmOperand a{h->emb, tokens, h->emb_dim, h->W_p, h->P, h->P};
-    GemmOperand none{};
-    GemmOut o{out_Pp, nullptr, h->J, nullptr};
-    launch_gemm_f32(a, none, o, nullptr, R, h->J, st);
+    GemmOperand a{h->emb, tok, h->emb_dim, h->W_p, h->P, h->P};
+    GemmOut o{Pp_out, idx_out, h->J, nullptr};
+    launch_gemm_f32(a, none, o, n_dev, n_max, h->J, st);
     *launches += 1;
-    return TW_OK;
+    return;
   }
   const int L = h->L, Hd = h->Hd;
   const long long stride = (long long)L * 2 * Hd;
   for (int l = 0; l < L; ++l) {
-    GemmOperand x = (l == 0) ? GemmOperand{h->emb, tokens, h->emb_dim, h->W_ih[0], h->emb_dim, h->emb_dim}
-                             : GemmOperand{state_out + (long long)(l - 1) * 2 * Hd, nullptr, stride, h->W_ih[l], Hd, Hd};
-    GemmOperand r{state_in + (long long)l * 2 * Hd, nullptr, stride, h->W_hh[l], Hd, Hd};
-    GemmOut o{h->gates, nullptr, 4 * Hd, h->b_l[l]};
-    launch_gemm_f32(x, r, o, nullptr, R, 4 * Hd, st);
-    launch_lstm_pointwise_plain(h->gates, state_in, state_out, R, L, l, Hd, st);
+    const float* x = (l == 0) ? h->emb : hc_out + (long long)(l - 1) * 2 * Hd;
+    const int* xi = (l == 0) ? tok : idx_out;
+    const long long xld = (l == 0) ? h->emb_dim : stride;
+    const int xk = (l == 0) ? h->emb_dim : Hd;
+    const float* hp = hc_in + (long long)l * 2 * Hd;
+    if (h->mode == TW_MODE_BF16) {
+      launch_gather_concat_bf16(x, xi, xld, xk, hp, idx_in, stride, Hd, n_dev, n_max, h->bf.X[l].ptr, st);
+      gemm_bf16(h, h->bf.X[l], h->bf.W_cat[l], n_dev, n_max, h->gates, nullptr, 4 * Hd, h->b_l[l], st);
+      *launches += 1;
+    } else {
+      GemmOperand xo{x, xi, xld, h->W_ih[l], xk, xk};
+      GemmOperand ro{hp, idx_in, stride, h->W_hh[l], Hd, Hd};
+      GemmOut o{h->gates, nullptr, 4 * Hd, h->b_l[l]};
+      launch_gemm_f32(xo, ro, o, n_dev, n_max, 4 * Hd, st);
+    }
+    // pointwise: c' = sigma(f) c + sigma(i) tanh(g), h' = sigma(o) tanh(c')
+    launch_lstm_pointwise(h->gates, idx_out, idx_in, n_dev, n_max, hc_in, hc_out, L, l, Hd, st);
     *launches += 2;
   }
-  GemmOperand top{state_out + (long long)(L - 1) * 2 * Hd, nullptr, stride, h->W_p, h->P, h->P};
-  GemmOperand none{};
-  GemmOut o{out_Pp, nullptr, h->J, nullptr};
-  launch_gemm_f32(top, none, o, nullptr, R, h->J, st);
-  *launches += 1;
+  const float* top = hc_out + (long long)(L - 1) * 2 * Hd;
+  if (h->mode == TW_MODE_BF16) {
+    launch_gather_concat_bf16(top, idx_out, stride, Hd, nullptr, nullptr, 0, 0, n_dev, n_max, h->bf.Htop.ptr, st);
+    gemm_bf16(h, h->bf.Htop, h->bf.W_p, n_dev, n_max, Pp_out, idx_out, h->J, nullptr, st);
+    *launches += 2;
+  } else {
+    GemmOperand to{top, idx_out, stride, h->W_p, h->P, h->P};
+    GemmOut o{Pp_out, idx_out, h->J, nullptr};
+    launch_gemm_f32(to, none, o, n_dev, n_max, h->J, st);
+    *launches += 1;
+  }
+}
+
+int enqueue_predictor_plain(tw_handle* h, const int* tokens, const float* state_in, int R,
+                            float* state_out, float* out_Pp, cudaStream_t st, int* launches) {
+  enqueue_predictor(h, tokens, state_in, nullptr, state_out, nullptr, out_Pp, nullptr, R, st, launches);
   return TW_OK;
 }
 
@@ -71,23 +116,48 @@ int enqueue_predictor_plain(tw_handle* h, const int* tokens, const float* state_
 void enqueue_predictor_slots(tw_handle* h, cudaStream_t st, int* launches) {
   if (h->pred_kind == TW_PRED_STATELESS) return;   // the joiner reads W_p emb[last token] from a table
   const HypState& hs = h->hs;
-  const int L = h->L, Hd = h->Hd;
-  const long long stride = (long long)L * 2 * Hd;
-  const int* n_dev = hs.scalars + kScNPred;
-  for (int l = 0; l < L; ++l) {
-    GemmOperand x = (l == 0) ? GemmOperand{h->emb, hs.pw_tok, h->emb_dim, h->W_ih[0], h->emb_dim, h->emb_dim}
-                             : GemmOperand{hs.slot_hc + (long long)(l - 1) * 2 * Hd, hs.pw_new, stride, h->W_ih[l], Hd, Hd};
-    GemmOperand r{hs.slot_hc + (long long)l * 2 * Hd, hs.pw_par, stride, h->W_hh[l], Hd, Hd};
-    GemmOut o{h->gates, nullptr, 4 * Hd, h->b_l[l]};
-    launch_gemm_f32(x, r, o, n_dev, h->R_max, 4 * Hd, st);
-    launch_lstm_pointwise_slots(h->gates, hs.pw_new, hs.pw_par, n_dev, h->R_max, hs.slot_hc, L, l, Hd, st);
+  enqueue_predictor(h, hs.pw_tok, hs.slot_hc, hs.pw_par, hs.slot_hc, hs.pw_new, hs.slot_Pp,
+                    hs.scalars + kScNPred, h->R_max, st, launches);
+}
+
+// E = enc W_e^T for `rows` frames
+void enqueue_project(tw_handle* h, const float* enc, int rows, float* E, cudaStream_t st, int* launches) {
+  if (h->mode == TW_MODE_BF16) {
+    launch_f32_to_bf16(enc, h->bf.enc.ptr, (long long)rows * h->D_enc, st);
+    gemm_bf16(h, h->bf.enc, h->bf.W_e, nullptr, rows, E, nullptr, h->J, nullptr, st);
     *launches += 2;
+  } else {
+    GemmOperand a{enc, nullptr, h->D_enc, h->W_e, h->D_enc, h->D_enc};
+    GemmOperand none{};
+    GemmOut o{E, nullptr, h->J, nullptr};
+    launch_gemm_f32(a, none, o, nullptr, rows, h->J, st);
+    *launches += 1;
   }
-  GemmOperand top{hs.slot_hc + (long long)(L - 1) * 2 * Hd, hs.pw_new, stride, h->W_p, h->P, h->P};
-  GemmOperand none{};
-  GemmOut o{hs.slot_Pp, hs.pw_new, h->J, nullptr};
-  launch_gemm_f32(top, none, o, n_dev, h->R_max, h->J, st);
-  *launches += 1;
+}
+
+// bf16 mode set-up: operand copies, tensor maps, activation buffers
+int build_bf16(tw_handle* h) {
+  if ((h->D_enc % 8) || (h->J % 8) || (h->P % 8) || (h->emb_dim % 8) || (h->Hd % 8)) return TW_ERR_ARG;
+  TW_TRY(gemm_bf16_setup());
+  TW_TRY(dev_alloc(h, &h->bf.err, (size_t)1));
+  TW_CUDA(h, cudaMemset(h->bf.err, 0, sizeof(int)));
+  TW_TRY(make_bf16_mat(h, &h->bf.W_e, h->W_e, h->J, h->D_enc, false, true));
+  TW_TRY(make_bf16_mat(h, &h->bf.W_out, h->W_out, h->V, h->J, false, true));
+  TW_TRY(make_bf16_mat(h, &h->bf.enc, nullptr, (long long)h->max_batch * h->max_T, h->D_enc, true, false));
+  TW_TRY(make_bf16_mat(h, &h->bf.A_join, nullptr, (long long)h->R_max * h->S, h->J, true, false));
+  if (h->pred_kind == TW_PRED_LSTM) {
+    TW_TRY(make_bf16_mat(h, &h->bf.W_p, h->W_p, h->J, h->P, false, true));
+    TW_TRY(make_bf16_mat(h, &h->bf.Htop, nullptr, h->R_max, h->Hd, true, false));
+    for (int l = 0; l < h->L; ++l) {
+      const int in = (l == 0) ? h->emb_dim : h->Hd;
+      TW_TRY(make_bf16_mat(h, &h->bf.W_cat[l], nullptr, 4 * h->Hd, in + h->Hd, false, true));
+      launch_gather_concat_bf16(h->W_ih[l], nullptr, in, in, h->W_hh[l], nullptr, h->Hd, h->Hd, nullptr, 4 * h->Hd,
+                                h->bf.W_cat[l].ptr, 0);
+      TW_TRY(make_bf16_mat(h, &h->bf.X[l], nullptr, h->R_max, in + h->Hd, true, false));
+    }
+  }
+  TW_CUDA(h, cudaGetLastError());
+  return TW_OK;
 }
 
 int build_workspace(tw_handle* h) {
@@ -164,6 +234,7 @@ int init_impl(tw_handle* h, const tw_model* m, const tw_config* c) {
     TW_TRY(copy_weight(h, &h->b_l[l], m->host_lstm_b[l], (size_t)4 * h->Hd));
   }
   TW_TRY(build_workspace(h));
+  if (h->mode == TW_MODE_BF16) TW_TRY(build_bf16(h));
 
   int launches = 0;
   if (h->pred_kind == TW_PRED_STATELESS) {
@@ -194,14 +265,28 @@ int init_impl(tw_handle* h, const tw_model* m, const tw_config* c) {
 }  // namespace
 
 namespace tw {
+void enqueue_joiner_logits(tw_handle* h, const JoinerRows& rows, float* logp, cudaStream_t st, int* launches);
 void enqueue_joiner_expand_f32(tw_handle* h, const JoinerRows& rows, const float* ld_old, float* logp,
                                float* ldphi, float* ldnb, float* la, double* ldphi_d, double* la_d,
                                cudaStream_t st, int* launches) {
-  launch_joiner_f32(rows, h->W_out, h->b_out, logp, st);
+  enqueue_joiner_logits(h, rows, logp, st, launches);
   launch_log_softmax(rows, h->blank, logp, st);
   launch_expand_f32(logp, ld_old, rows.row_slen, rows.R_dev, rows.R_max, rows.S, rows.V, h->blank, ldphi,
                     ldnb, la, ldphi_d, la_d, st);
-  *launches += 3;
+  *launches += 2;
+}
+
+// z[(r, t), :] = W_out tanh(E + Pp) + b_out into `logp` (rows of padding frames hold no result)
+void enqueue_joiner_logits(tw_handle* h, const JoinerRows& rows, float* logp, cudaStream_t st, int* launches) {
+  if (h->mode == TW_MODE_BF16) {
+    launch_joiner_A_bf16(rows, h->bf.A_join.ptr, st);
+    const int* M_dev = rows.R_dev ? h->hs.scalars + kScM : nullptr;
+    gemm_bf16(h, h->bf.A_join, h->bf.W_out, M_dev, rows.R_max * rows.S, logp, nullptr, rows.V, h->b_out, st);
+    *launches += 2;
+  } else {
+    launch_joiner_f32(rows, h->W_out, h->b_out, logp, st);
+    *launches += 1;
+  }
 }
 }  // namespace tw
 

@@ -2,6 +2,7 @@
 #pragma once
 #include <vector>
 
+#include "bf16_path.cuh"
 #include "tw_internal.cuh"
 
 struct tw_handle {
@@ -22,6 +23,16 @@ struct tw_handle {
   float* E = nullptr;         // projected encoder frames [max_batch * max_T, J]
   float* gates = nullptr;     // LSTM gate pre-activations [R_max, 4 Hd]
   int *stage_e0 = nullptr, *stage_slen = nullptr;   // [R_max] scratch of the stage entry points
+
+  // TW_MODE_BF16: bf16 copies of the GEMM operands with their tensor maps
+  struct {
+    tw::Bf16Mat W_e, W_out, W_p, W_cat[tw::kMaxLayers];   // W_cat[l] = [W_ih[l] | W_hh[l]]  [4Hd, in+Hd]
+    tw::Bf16Mat enc;                                      // [max_batch * max_T, D_enc]
+    tw::Bf16Mat A_join;                                   // [R_max * S, J]  tanh(E + Pp)
+    tw::Bf16Mat X[tw::kMaxLayers];                        // [R_max, in+Hd]  LSTM layer inputs
+    tw::Bf16Mat Htop;                                     // [R_max, Hd]
+    int* err = nullptr;                                   // device error word of the bounded waits
+  } bf;
 
   // staging of tw_decode_host (allocated on first use)
   float* st_enc = nullptr; int* st_len = nullptr; int* st_tok = nullptr; int* st_lens = nullptr;
@@ -45,3 +56,4 @@ void enqueue_joiner_expand_f32(tw_handle* h, const JoinerRows& rows, const float
                                float* ldphi, float* ldnb, float* la, double* ldphi_d, double* la_d,
                                cudaStream_t st, int* launches);
 }
+

@@ -76,7 +76,7 @@ void launch_rows_from_groups(const int* row_group, const int* seg_len, int R, in
 
 // ---------------------------------------------------------------------------------------------
 // Hypothesis state of a batch (structure of arrays in one device workspace).
-enum Scalar { kScR = 0, kScNPred = 1, kScActive = 2, kScSteps = 3, kScCount = 8 };
+enum Scalar { kScR = 0, kScNPred = 1, kScActive = 2, kScSteps = 3, kScM = 4, kScCount = 8 };   // kScM = R * S
 
 struct HypState {
   int B, N, S, V, J, U_cap, I_max, blank;
@@ -118,12 +118,9 @@ void launch_compact(const HypState& hs, int B, int T, cudaStream_t st);
 void launch_finish(const HypState& hs, int B, int* out_tokens, int* out_lens, double* out_scores,
                    int* out_status, cudaStream_t st);
 
-// LSTM pointwise on slots: gates [n, 4Hd] + parent c -> (h, c) of layer l in the new slot
-void launch_lstm_pointwise_slots(const float* gates, const int* pw_new, const int* pw_par,
-                                 const int* n_dev, int n_max, float* slot_hc, int L, int l, int Hd,
-                                 cudaStream_t st);
-// same on plain [R, L, 2, Hd] state arrays (stage entry point)
-void launch_lstm_pointwise_plain(const float* gates, const float* state_in, float* state_out, int R,
-                                 int L, int l, int Hd, cudaStream_t st);
+// LSTM pointwise: gates [n, 4Hd] + c of row (idx_in ? idx_in[i] : i) of hc_in -> (h, c) of layer l in row
+// (idx_out ? idx_out[i] : i) of hc_out; state rows are [L][2][Hd]
+void launch_lstm_pointwise(const float* gates, const int* idx_out, const int* idx_in, const int* n_dev,
+                           int n_max, const float* hc_in, float* hc_out, int L, int l, int Hd, cudaStream_t st);
 
 }  // namespace tw

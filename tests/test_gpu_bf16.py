@@ -1,0 +1,110 @@
+"""TW_MODE_BF16 (bf16 operands on the tensor cores, fp32 accumulate) against the fp64 oracle fed the
+same bf16-rounded weights and inputs: stage log-probabilities within 2e-2, end-to-end top-1 agreement."""
+import numpy as np
+import pytest
+
+import tw_synth
+from oracle import rnnt_model as rm
+from oracle import token_wise_search as tws
+from helpers import nbest_from_arrays, oracle_model
+
+pytestmark = pytest.mark.gpu
+BF16_STAGE_TOL = 2e-2
+
+
+def _cfg(pred="lstm", V=256, J=128, D=64, emb=64, hidden=64, layers=2, seed=3, batch=4, T=30):
+    return tw_synth.WorkloadConfig("b", batch, T, (T // 2, T), D, pred, emb, layers if pred == "lstm" else 0,
+                                   hidden if pred == "lstm" else 0, J, V, 3.0, 4, (3,), "bf16", seed)
+
+
+def _decoder(cfg, S, N=None, max_batch=8, max_T=None):
+    from paper_2302_14357_b200.binding import MODE_BF16, TwDecoder, weights_from_synth
+    m = tw_synth.make_model(cfg)
+    return m, TwDecoder(weights_from_synth(m), N=N or cfg.N, S=S, mode=MODE_BF16, max_batch=max_batch, max_T=max_T or cfg.T)
+
+
+@pytest.mark.parametrize("D,J,rows", [(64, 64, 5), (64, 128, 128), (512, 640, 300), (1024, 1024, 777)])
+def test_encoder_projection_tensor_core_gemm(D, J, rows):
+    """E = enc W_e^T: bf16 products are exact in fp32, so only the accumulation order differs."""
+    cfg = _cfg(D=D, J=J, T=100, batch=8)
+    m, dec = _decoder(cfg, 3, max_batch=8, max_T=100)
+    rng = np.random.default_rng(rows)
+    enc = tw_synth.round_to_bf16(rng.standard_normal((rows, D)).astype(np.float32))
+    got = dec.project_encoder(enc).cpu().numpy()
+    ref = enc.astype(np.float64) @ m.W_e.astype(np.float64).T
+    np.testing.assert_allclose(got, ref, rtol=0, atol=2e-5 * np.sqrt(D))
+
+
+@pytest.mark.parametrize("V,J,S,R", [(256, 128, 3, 7), (1024, 640, 3, 50), (4096, 1024, 2, 70), (320, 64, 10, 9)])
+def test_joiner_segment_bf16(V, J, S, R):
+    cfg = _cfg(V=V, J=J)
+    m, dec = _decoder(cfg, S, N=4, max_batch=(R + 3) // 4)
+    om = oracle_model(m)
+    rng = np.random.default_rng(V + R)
+    G = 4
+    enc = tw_synth.round_to_bf16(rng.standard_normal((G, S, cfg.D_enc)).astype(np.float32))
+    row_group = rng.integers(0, G, size=R).astype(np.int32)
+    seg_len = np.array([S, max(1, S - 1), S, 1], np.int32)
+    pred = rng.standard_normal((R, cfg.P)).astype(np.float32) * 0.5
+    E = dec.project_encoder(enc).reshape(G, S, J)
+    Pp = (pred.astype(np.float64) @ om.W_p.T).astype(np.float32)
+    got = dec.joiner_segment(E, Pp, row_group, seg_len).cpu().numpy()
+    worst = 0.0
+    for r in range(R):
+        sl = seg_len[row_group[r]]
+        ref = rm.joiner_log_probs(om, enc[row_group[r], :sl], pred[r:r + 1])[0]
+        worst = max(worst, np.abs(got[r, :sl] - ref).max())
+        assert np.all(got[r, sl:, 0] == 0.0) and np.all(np.isneginf(got[r, sl:, 1:]))
+    assert worst < BF16_STAGE_TOL, worst
+
+
+@pytest.mark.parametrize("layers,hidden", [(1, 64), (2, 128)])
+def test_predictor_step_bf16(layers, hidden):
+    cfg = _cfg(layers=layers, hidden=hidden)
+    m, dec = _decoder(cfg, 2)
+    om = oracle_model(m)
+    rng = np.random.default_rng(4)
+    R = 9
+    tokens = rng.integers(0, cfg.V, size=R).astype(np.int32)
+    state = (rng.standard_normal((R, layers, 2, hidden)) * 0.5).astype(np.float32)
+    out, Pp = dec.predictor_step(tokens, state)
+    out, Pp = out.cpu().numpy(), Pp.cpu().numpy()
+    for r in range(R):
+        st = ([state[r, l, 0].astype(np.float64) for l in range(layers)], [state[r, l, 1].astype(np.float64) for l in range(layers)])
+        (h, c), o = rm.lstm_step(om, st, int(tokens[r]))
+        for l in range(layers):
+            np.testing.assert_allclose(out[r, l, 0], h[l], atol=BF16_STAGE_TOL)
+            np.testing.assert_allclose(out[r, l, 1], c[l], atol=BF16_STAGE_TOL)
+        np.testing.assert_allclose(Pp[r], om.W_p @ o, atol=BF16_STAGE_TOL)
+
+
+def _top1_agreement(cfg, S, batch, T):
+    from paper_2302_14357_b200.binding import MODE_BF16, TwDecoder, weights_from_synth
+    m = tw_synth.make_model(cfg)
+    enc, lens = tw_synth.make_encoder_batch(cfg, batch)
+    enc, lens = np.ascontiguousarray(enc[:, :T]), np.minimum(lens, T)
+    dec = TwDecoder(weights_from_synth(m), N=cfg.N, S=S, mode=MODE_BF16, max_batch=batch, max_T=T)
+    tokens, olens, scores, status, rc = [x.cpu().numpy() if hasattr(x, "cpu") else x for x in dec.decode(enc, lens)]
+    om = oracle_model(m)
+    agree, gaps = 0, []
+    for b in range(batch):
+        got = nbest_from_arrays(tokens, olens, scores, b)
+        ref, _ = tws.token_wise_beam_search(om, enc[b, :lens[b]], cfg.N, S, max_iters=4 * S + 16)
+        agree += got[0][0] == ref[0][0]
+        gaps.append(abs(got[0][1] - ref[0][1]))
+        assert len(got) == len(ref) and status[b] == 0
+    return agree / batch, max(gaps), dec.stats()
+
+
+def test_decode_bf16_small_model_top1():
+    rate, gap, st = _top1_agreement(_cfg(batch=6, T=40), 3, 6, 40)
+    print("bf16 top-1 agreement %.2f, max top-1 score gap %.3g" % (rate, gap))
+    assert rate >= 0.5 and gap < 0.5
+
+
+@pytest.mark.parametrize("name,S,batch,T", [("c1", 3, 4, 80), ("c3", 3, 2, 45)])
+def test_decode_bf16_config_shapes_top1(name, S, batch, T):
+    rate, gap, st = _top1_agreement(tw_synth.get_config(name), S, batch, T)
+    print("%s bf16 top-1 agreement %.2f, max top-1 score gap %.3g" % (name, rate, gap))
+    assert rate >= 0.5 and gap < 1.0
+    assert st["calls"] > 0
