@@ -174,7 +174,7 @@ def run_ours(args, cfg, S):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
-    mode_name = "f32" if args.mode == "auto" else args.mode
+    mode_name = cfg.dtype if args.mode == "auto" else args.mode
     mode = MODE_BF16 if mode_name == "bf16" else MODE_F32
     B = args.batch or cfg.batch
     model = tw_synth.make_model(cfg)
