@@ -23,18 +23,6 @@ __device__ __forceinline__ unsigned long long hash_push(unsigned long long h, in
   return x;
 }
 
-__device__ __forceinline__ int block_min_int(int v, int* scratch) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v = min(v, __shfl_xor_sync(0xffffffffu, v, o));
-  __syncthreads();
-  if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
-  __syncthreads();
-  int r = scratch[0];
-#pragma unroll
-  for (int i = 1; i < kThreads / 32; ++i) r = min(r, scratch[i]);
-  return r;
-}
-
 // Starts the next segment of utterance b: A = ChooseNBest(B), B = [], t += S, d = (s, 0, ..., 0).
 // Precondition: list A is empty and frames remain.  Called by the whole CTA.
 __device__ void turn_over(const HypState& hs, int b) {
@@ -97,25 +85,19 @@ __global__ void __launch_bounds__(kThreads) hyp_init_kernel(HypState hs, const i
   if (hs.len[b] > 0) turn_over(hs, b);
 }
 
-__device__ __forceinline__ bool better(float v, int k, float v2, int k2) {
-  return v > v2 || (v == v2 && k < k2);
-}
+constexpr int kStepThreads = 512;   // 16 warps: one per hypothesis of list A
 
-__global__ void __launch_bounds__(kThreads) hyp_step_kernel(HypState hs) {
-  __shared__ int s_scratch[kThreads / 32];
-  __shared__ int s_nB, s_hasthr, s_nkeep, s_ntot;
-  __shared__ int s_touched[kMaxBeam];
+__global__ void __launch_bounds__(kStepThreads) hyp_step_kernel(HypState hs) {
+  __shared__ int s_nB, s_hasthr, s_nkeep;
+  __shared__ int s_found[kMaxBeam], s_touched[kMaxBeam], s_carry[kMaxBeam];
   __shared__ double s_Als[kMaxBeam];
   __shared__ int s_Aslot[kMaxBeam];
   __shared__ double s_thr;
-  __shared__ float s_cv[kMaxBeam][kMaxBeam];
-  __shared__ int s_ck[kMaxBeam][kMaxBeam];
-  __shared__ int s_cnt[kMaxBeam];
+  __shared__ int s_ck[kMaxBeam * kMaxBeam];
   __shared__ double s_abs[kMaxBeam * kMaxBeam];
   __shared__ int s_sel[kMaxBeam];
   __shared__ int s_keep_h[kMaxBeam], s_keep_k[kMaxBeam], s_keep_slot[kMaxBeam];
   __shared__ double s_keep_ls[kMaxBeam];
-  __shared__ double s_newld[kMaxBeam][kMaxSeg];
 
   const int b = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -124,56 +106,67 @@ __global__ void __launch_bounds__(kThreads) hyp_step_kernel(HypState hs) {
   const int N = hs.N, S = hs.S, V = hs.V;
   const int r0 = hs.row_off[b];
   const int slen = hs.slen[b];
+  const int nB0 = hs.nB[b];
   const long long bB = (long long)b * hs.capB;
   const long long bS = (long long)b * hs.capSlot;
 
-  if (tid < H) { s_Als[tid] = hs.A_ls[b * kMaxBeam + tid]; s_Aslot[tid] = hs.A_slot[b * kMaxBeam + tid]; }
-  if (tid == 0) {
-    s_nB = hs.nB[b];
-    hs.calls[b] += 1;
-    hs.joins[b] += slen;
+  if (tid < kMaxBeam) {
+    if (tid < H) { s_Als[tid] = hs.A_ls[b * kMaxBeam + tid]; s_Aslot[tid] = hs.A_slot[b * kMaxBeam + tid]; }
+    s_carry[tid] = hs.carry[b * kMaxBeam + tid];
   }
+  if (tid == 0) { hs.calls[b] += 1; hs.joins[b] += slen; }
   __syncthreads();
 
-  // ---- AddAndMerge of the blank expansions (tok, delta_phi, o) into list B -------------------
-  for (int h = 0; h < H; ++h) {
-    const int slot = s_Aslot[h];
+  // ---- AddAndMerge, search: warp h looks for the tokens of A_h among the entries already in B.
+  // (Entries of A are distinct sequences, so two of them never merge with each other.)
+  if (warp < H) {
+    const int slot = s_Aslot[warp];
     const unsigned long long hh = hs.slot_hash[bS + slot];
     const int ln = hs.slot_len[bS + slot];
-    const int nB = s_nB;
-    int start = 0, found = -1;
-    while (true) {
-      int local = 0x7fffffff;
-      for (int e = start + tid; e < nB; e += kThreads) {
-        if (hs.B_hash[bB + e] == hh && hs.B_len[bB + e] == ln) { local = e; break; }
-      }
-      const int cand = block_min_int(local, s_scratch);
-      if (cand == 0x7fffffff) break;
-      // verify token by token (a 64-bit hash match is not proof)
-      const int oslot = hs.B_slot[bB + cand];
-      int diff = 0;
-      if (oslot != slot) {
-        const int* ta = hs.slot_tok + (bS + slot) * hs.U_cap;
-        const int* tb = hs.slot_tok + (bS + oslot) * hs.U_cap;
-        for (int i = tid; i < ln; i += kThreads) diff |= (ta[i] != tb[i]);
-      }
-      if (!__syncthreads_or(diff)) { found = cand; break; }
-      start = cand + 1;
-    }
-    if (tid == 0) {
-      const double val = s_Als[h] + (hs.ldphi_d ? hs.ldphi_d[r0 + h] : (double)hs.ldphi[r0 + h]);
-      if (found >= 0) {
-        hs.B_ls[bB + found] = logaddexp_d(hs.B_ls[bB + found], val);
-        s_touched[h] = found;
-      } else {
-        const int e = s_nB;                 // capB = N * I_max bounds this by construction
-        hs.B_slot[bB + e] = slot; hs.B_ls[bB + e] = val; hs.B_hash[bB + e] = hh; hs.B_len[bB + e] = ln;
-        s_touched[h] = e;
-        s_nB = e + 1;
+    const int* ta = hs.slot_tok + (bS + slot) * hs.U_cap;
+    int found = -1;
+    for (int base = 0; base < nB0 && found < 0; base += 32) {
+      const int e = base + lane;
+      const bool match = e < nB0 && hs.B_hash[bB + e] == hh && hs.B_len[bB + e] == ln;
+      unsigned mask = __ballot_sync(0xffffffffu, match);
+      while (mask != 0 && found < 0) {
+        const int c = base + __ffs(mask) - 1;
+        mask &= mask - 1;
+        const int oslot = hs.B_slot[bB + c];
+        int diff = 0;                       // a 64-bit hash match is not proof: compare the tokens
+        if (oslot != slot) {
+          const int* tb = hs.slot_tok + (bS + oslot) * hs.U_cap;
+          for (int i = lane; i < ln; i += 32) diff |= (ta[i] != tb[i]);
+        }
+        if (!__any_sync(0xffffffffu, diff)) found = c;
       }
     }
-    __syncthreads();
+    if (lane == 0) s_found[warp] = found;
   }
+  __syncthreads();
+  // ---- AddAndMerge, apply: sum into the matching entry or append (appends keep the order of A)
+  if (tid < H) {
+    const int h = tid;
+    const int slot = s_Aslot[h];
+    const double val = s_Als[h] + (hs.ldphi_d ? hs.ldphi_d[r0 + h] : (double)hs.ldphi[r0 + h]);
+    int e = s_found[h];
+    if (e >= 0) {
+      hs.B_ls[bB + e] = logaddexp_d(hs.B_ls[bB + e], val);
+    } else {
+      e = nB0;                              // capB = N * I_max bounds this by construction
+      for (int q = 0; q < h; ++q) e += (s_found[q] < 0);
+      hs.B_slot[bB + e] = slot; hs.B_ls[bB + e] = val;
+      hs.B_hash[bB + e] = hs.slot_hash[bS + slot]; hs.B_len[bB + e] = hs.slot_len[bS + slot];
+    }
+    s_touched[h] = e;
+  }
+  if (tid == 0) {
+    int nB = nB0;
+    for (int q = 0; q < H; ++q) nB += (s_found[q] < 0);
+    s_nB = nB;
+    hs.nB[b] = nB;
+  }
+  __syncthreads();
 
   // ---- ChooseNthScore: the best N of B are among the previous best N and the entries touched now
   if (warp == 0) {
@@ -198,99 +191,41 @@ __global__ void __launch_bounds__(kThreads) hyp_step_kernel(HypState hs) {
     __syncwarp();
     if (idx >= 0 && rank < N) hs.B_top[b * kMaxBeam + rank] = idx;
     if (idx >= 0 && rank == N - 1) s_thr = score;
-    if (lane == 0) {
-      hs.nTop[b] = min(N, count);
-      s_hasthr = (count >= N);
-      hs.nB[b] = s_nB;
+    if (lane == 0) { hs.nTop[b] = min(N, count); s_hasthr = (count >= N); }
+  }
+  // ---- ChooseNBestExpansions, second stage: the N best (h, k) over the rows' candidate lists, in
+  // float64; order (score desc, h asc, k asc).  The lists are sorted by (score desc, k asc).
+  if (tid < kMaxBeam * kMaxBeam) {
+    const int h = tid / kMaxBeam, j = tid % kMaxBeam;
+    const bool valid = h < H && j < hs.cand_n[r0 + h];
+    s_abs[tid] = valid ? s_Als[h] + (double)hs.cand_v[(long long)(r0 + h) * kMaxBeam + j] : -INFINITY;
+    s_ck[tid] = valid ? hs.cand_k[(long long)(r0 + h) * kMaxBeam + j] : -1;
+  }
+  if (tid < kMaxBeam) s_sel[tid] = -1;
+  __syncthreads();
+  if (tid < kMaxBeam * kMaxBeam && s_ck[tid] >= 0) {
+    const double mine = s_abs[tid];
+    int rank = 0;
+    for (int o = 0; o < kMaxBeam * kMaxBeam; ++o) {
+      const double so = s_abs[o];
+      if (s_ck[o] >= 0 && (so > mine || (so == mine && o < tid))) ++rank;
     }
+    if (rank < N) s_sel[rank] = tid;
   }
   __syncthreads();
   const bool hasthr = s_hasthr != 0;
   const double thr = hasthr ? s_thr : -INFINITY;
 
-  // ---- ChooseNBestExpansions, stage 1: per hypothesis row, the N best non-blank tokens -------
-  for (int h = warp; h < H; h += kThreads / 32) {
-    const float* row = hs.ldnb + (long long)(r0 + h) * V;
-    // anything at or below the threshold fails the filter later; a small slack keeps the exact
-    // float64 comparison authoritative
-    const float bound = hasthr ? (float)(thr - s_Als[h]) - 1e-3f : -INFINITY;
-    float lv[kMaxBeam]; int lk[kMaxBeam];
-#pragma unroll
-    for (int j = 0; j < kMaxBeam; ++j) { lv[j] = -INFINITY; lk[j] = 0x7fffffff; }
-    float admit = bound;
-    for (int k = lane; k < V; k += 32) {
-      const float v = row[k];               // the blank column holds -inf and never passes
-      if (v > admit) {
-        float cv = v; int ck = k;
-#pragma unroll
-        for (int j = 0; j < kMaxBeam; ++j) {
-          if (better(cv, ck, lv[j], lk[j])) {
-            const float tv = lv[j]; const int tk = lk[j];
-            lv[j] = cv; lk[j] = ck; cv = tv; ck = tk;
-          }
-        }
-        float last = -INFINITY;
-#pragma unroll
-        for (int j = 0; j < kMaxBeam; ++j) if (j == N - 1) last = lv[j];
-        admit = fmaxf(bound, last);
-      }
-    }
-    int cnt = 0;
-    for (int j = 0; j < N; ++j) {
-      float bv = lv[0]; int bk = lk[0]; int bl = lane;
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-        const int ok = __shfl_xor_sync(0xffffffffu, bk, o);
-        const int ol = __shfl_xor_sync(0xffffffffu, bl, o);
-        if (better(ov, ok, bv, bk)) { bv = ov; bk = ok; bl = ol; }
-      }
-      if (bv == -INFINITY) break;
-      if (lane == 0) { s_cv[h][j] = bv; s_ck[h][j] = bk; }
-      if (lane == bl) {
-#pragma unroll
-        for (int i = 0; i < kMaxBeam - 1; ++i) { lv[i] = lv[i + 1]; lk[i] = lk[i + 1]; }
-        lv[kMaxBeam - 1] = -INFINITY; lk[kMaxBeam - 1] = 0x7fffffff;
-      }
-      ++cnt;
-    }
-    if (lane == 0) s_cnt[h] = cnt;
-  }
-  __syncthreads();
-
-  // ---- stage 2: the N best (h, k) over all rows, in float64; order (score desc, h asc, k asc) -
-  {
-    const int h = tid / kMaxBeam, j = tid % kMaxBeam;
-    const bool valid = h < H && j < s_cnt[h];
-    s_abs[tid] = valid ? s_Als[h] + (double)s_cv[h][j] : -INFINITY;
-    if (tid == 0) s_ntot = 0;
-    __syncthreads();
-    if (valid) {
-      const double mine = s_abs[tid];
-      int rank = 0;
-      for (int o = 0; o < kMaxBeam * kMaxBeam; ++o) {
-        const int oh = o / kMaxBeam, oj = o % kMaxBeam;
-        if (oh < H && oj < s_cnt[oh]) {
-          const double so = s_abs[o];
-          if (so > mine || (so == mine && o < tid)) ++rank;   // o < tid  <=>  (h, k) order: rows are sorted by (v desc, k asc)
-        }
-      }
-      if (rank < N) s_sel[rank] = tid;
-      atomicAdd(&s_ntot, 1);
-    }
-    __syncthreads();
-  }
-
   // ---- filter against the threshold, allocate slots ------------------------------------------
   if (tid == 0) {
-    const int nC = min(N, s_ntot);
     int nk = 0;
     int cur = hs.cursor[b];
     const bool capped = hs.iters[b] + 1 >= hs.I_max;
     hs.iters[b] += 1;
-    for (int i = 0; i < nC; ++i) {
+    for (int i = 0; i < N; ++i) {
       const int c = s_sel[i];
-      const int h = c / kMaxBeam, j = c % kMaxBeam;
+      if (c < 0) break;
+      const int h = c / kMaxBeam;
       const double sc = s_abs[c];
       if (hasthr && !(sc > thr)) continue;            // Length(B) < N or delta_nb > threshold
       if (capped) { hs.status[b] = TW_ERR_LIMIT; break; }
@@ -300,55 +235,48 @@ __global__ void __launch_bounds__(kThreads) hyp_step_kernel(HypState hs) {
       do {
         cur = (cur + 1 == hs.capSlot) ? 0 : cur + 1;
         busy = false;
-        for (int q = 0; q < kMaxBeam; ++q) busy |= (hs.carry[b * kMaxBeam + q] == cur);
+#pragma unroll
+        for (int q = 0; q < kMaxBeam; ++q) busy |= (s_carry[q] == cur);
       } while (busy);
-      s_keep_h[nk] = h; s_keep_k[nk] = s_ck[h][j]; s_keep_ls[nk] = sc; s_keep_slot[nk] = cur;
+      s_keep_h[nk] = h; s_keep_k[nk] = s_ck[c]; s_keep_ls[nk] = sc; s_keep_slot[nk] = cur;
       ++nk;
     }
     hs.cursor[b] = cur;
     s_nkeep = nk;
+    hs.nA[b] = nk; hs.n_new[b] = nk;
   }
   __syncthreads();
   const int nk = s_nkeep;
 
-  // ---- new list A: tokens, hash, frame distribution d_h(k) (Eq. 5) ----------------------------
-  for (int i = 0; i < nk; ++i) {
+  // ---- new list A (one warp per kept expansion): tokens, hash, frame distribution d_h(k) (Eq. 5)
+  if (warp < nk) {
+    const int i = warp;
     const int h = s_keep_h[i], k = s_keep_k[i];
     const long long gp = bS + s_Aslot[h], gn = bS + s_keep_slot[i];
     const int plen = hs.slot_len[gp];
     const int* src = hs.slot_tok + gp * hs.U_cap;
     int* dst = hs.slot_tok + gn * hs.U_cap;
-    for (int q = tid; q < plen; q += kThreads) dst[q] = src[q];
-    if (tid == 0) {
+    for (int q = lane; q < plen; q += 32) dst[q] = src[q];
+    if (lane == 0) {
       dst[plen] = k;
       hs.slot_len[gn] = plen + 1;
       hs.slot_hash[gn] = hash_push(hs.slot_hash[gp], k);
       hs.new_slot[b * kMaxBeam + i] = (int)gn;
       hs.new_par[b * kMaxBeam + i] = (int)gp;
       hs.new_tok[b * kMaxBeam + i] = k;
+      hs.A_slot[b * kMaxBeam + i] = s_keep_slot[i];
+      hs.A_ls[b * kMaxBeam + i] = s_keep_ls[i];
     }
-    if (tid < S) {
+    const long long r = r0 + h;
+    for (int t = lane; t < S; t += 32) {
       double v = -INFINITY;
-      if (tid < slen && hs.logp != nullptr) {
-        const long long r = r0 + h;
-        const double a = hs.la_d ? hs.la_d[r * S + tid] : (double)hs.la[r * S + tid];
-        v = s_Als[h] + a + (double)hs.logp[(r * S + tid) * V + k];
+      if (t < slen && hs.logp != nullptr) {
+        const double a = hs.la_d ? hs.la_d[r * S + t] : (double)hs.la[r * S + t];
+        v = s_Als[h] + a + (double)hs.logp[(r * S + t) * V + k];
       }
-      s_newld[i][tid] = v;
+      hs.A_ld[((long long)b * kMaxBeam + i) * S + t] = v;
     }
   }
-  __syncthreads();
-  if (tid < nk) {
-    hs.A_slot[b * kMaxBeam + tid] = s_keep_slot[tid];
-    hs.A_ls[b * kMaxBeam + tid] = s_keep_ls[tid];
-  }
-  for (int i = tid; i < nk * S; i += kThreads) {
-    const int a = i / S, t = i - a * S;
-    hs.A_ld[((long long)b * kMaxBeam + a) * S + t] = s_newld[a][t];
-  }
-  if (tid == 0) { hs.nA[b] = nk; hs.n_new[b] = nk; }
-  __syncthreads();
-
   // ---- list A empty: this segment is done ------------------------------------------------------
   if (nk == 0 && hs.t0[b] + slen < hs.len[b]) turn_over(hs, b);
 }
@@ -361,55 +289,60 @@ __global__ void __launch_bounds__(1024) compact_kernel(HypState hs, int B, int T
   const int tid = threadIdx.x;
   if (tid == 0) { s_base_a = 0; s_base_n = 0; s_frames = 0; }
   __syncthreads();
+  // exclusive scans of the list sizes -> row_off, new_off
   for (int b0 = 0; b0 < B; b0 += 1024) {
     const int b = b0 + tid;
     const int a = b < B ? hs.nA[b] : 0;
     const int nn = b < B ? hs.n_new[b] : 0;
     s_a[tid] = a; s_n[tid] = nn;
     __syncthreads();
-    for (int o = 1; o < 1024; o <<= 1) {          // inclusive scan
+    for (int o = 1; o < 1024; o <<= 1) {
       int va = 0, vn = 0;
       if (tid >= o) { va = s_a[tid - o]; vn = s_n[tid - o]; }
       __syncthreads();
       s_a[tid] += va; s_n[tid] += vn;
       __syncthreads();
     }
-    const int off_a = s_base_a + s_a[tid] - a;
-    const int off_n = s_base_n + s_n[tid] - nn;
     if (b < B) {
-      hs.row_off[b] = off_a;
-      const int t0 = hs.t0[b], sl = hs.slen[b];
-      if (a > 0) atomicAdd(&s_frames, a * sl);
-      for (int h = 0; h < a; ++h) {
-        const int r = off_a + h;
-        const int slot = hs.A_slot[b * kMaxBeam + h];
-        const long long gs = (long long)b * hs.capSlot + slot;
-        hs.row_b[r] = b;
-        hs.row_e0[r] = b * T + t0;
-        hs.row_slen[r] = sl;
-        if (hs.stateless) {
-          const int ln = hs.slot_len[gs];
-          hs.row_p[r] = ln > 0 ? hs.slot_tok[gs * hs.U_cap + ln - 1] : hs.blank;
-        } else {
-          hs.row_p[r] = (int)gs;
-        }
-        const double ls = hs.A_ls[b * kMaxBeam + h];
-        for (int t = 0; t < hs.S; ++t) {
-          const double d = hs.A_ld[((long long)b * kMaxBeam + h) * hs.S + t];
-          hs.row_ld[(long long)r * hs.S + t] = (d == -INFINITY) ? -INFINITY : (float)(d - ls);
-        }
-      }
-      for (int j = 0; j < nn; ++j) {
-        hs.pw_new[off_n + j] = hs.new_slot[b * kMaxBeam + j];
-        hs.pw_par[off_n + j] = hs.new_par[b * kMaxBeam + j];
-        hs.pw_tok[off_n + j] = hs.new_tok[b * kMaxBeam + j];
-      }
-      hs.n_new[b] = 0;
+      hs.row_off[b] = s_base_a + s_a[tid] - a;
+      hs.new_off[b] = s_base_n + s_n[tid] - nn;
+      if (a > 0) atomicAdd(&s_frames, a * hs.slen[b]);
     }
     __syncthreads();
     if (tid == 1023) { s_base_a += s_a[1023]; s_base_n += s_n[1023]; }
     __syncthreads();
   }
+  // fill: one thread per (utterance, list position)
+  for (int idx = tid; idx < B * kMaxBeam; idx += 1024) {
+    const int b = idx / kMaxBeam, h = idx % kMaxBeam;
+    if (h < hs.nA[b]) {
+      const int r = hs.row_off[b] + h;
+      const int slot = hs.A_slot[b * kMaxBeam + h];
+      const long long gs = (long long)b * hs.capSlot + slot;
+      hs.row_b[r] = b;
+      hs.row_e0[r] = b * T + hs.t0[b];
+      hs.row_slen[r] = hs.slen[b];
+      if (hs.stateless) {
+        const int ln = hs.slot_len[gs];
+        hs.row_p[r] = ln > 0 ? hs.slot_tok[gs * hs.U_cap + ln - 1] : hs.blank;
+      } else {
+        hs.row_p[r] = (int)gs;
+      }
+      const double ls = hs.A_ls[b * kMaxBeam + h];
+      for (int t = 0; t < hs.S; ++t) {
+        const double d = hs.A_ld[((long long)b * kMaxBeam + h) * hs.S + t];
+        hs.row_ld[(long long)r * hs.S + t] = (d == -INFINITY) ? -INFINITY : (float)(d - ls);
+      }
+    }
+    if (h < hs.n_new[b]) {
+      const int o = hs.new_off[b] + h;
+      hs.pw_new[o] = hs.new_slot[b * kMaxBeam + h];
+      hs.pw_par[o] = hs.new_par[b * kMaxBeam + h];
+      hs.pw_tok[o] = hs.new_tok[b * kMaxBeam + h];
+    }
+  }
+  __syncthreads();
+  for (int b = tid; b < B; b += 1024) hs.n_new[b] = 0;
   if (tid == 0) {
     const int R = s_base_a;
     hs.scalars[kScR] = R;
@@ -470,7 +403,7 @@ void launch_hyp_init(const HypState& hs, const int* lengths, int B, int T, cudaS
   if (B > 0) hyp_init_kernel<<<B, kThreads, 0, st>>>(hs, lengths, T);
 }
 void launch_hyp_step(const HypState& hs, int B, cudaStream_t st) {
-  if (B > 0) hyp_step_kernel<<<B, kThreads, 0, st>>>(hs);
+  if (B > 0) hyp_step_kernel<<<B, kStepThreads, 0, st>>>(hs);
 }
 void launch_compact(const HypState& hs, int B, int T, cudaStream_t st) {
   compact_kernel<<<1, 1024, 0, st>>>(hs, B, T);

@@ -1,5 +1,6 @@
 // fp32 (TW_MODE_F32) stage kernels: SIMT GEMM, joiner contraction, log-softmax, Eq. 3-7.
 // This is the accuracy path: plain FFMA accumulation and libm tanhf/expf/logf, no fast-math.
+#include "topn.cuh"
 #include "tw_internal.cuh"
 
 namespace tw {
@@ -194,8 +195,11 @@ __global__ void __launch_bounds__(256) expand_f32_kernel(const float* __restrict
                                                          const int* row_slen, const int* R_dev,
                                                          int R_max, int S, int V, int blank,
                                                          float* ldphi, float* ldnb, float* la_out,
-                                                         double* ldphi_d, double* la_d) {
+                                                         double* ldphi_d, double* la_d, CandOut cand) {
   __shared__ float la[kMaxSeg];
+  __shared__ float s_wv[8][kMaxBeam];
+  __shared__ int s_wk[8][kMaxBeam];
+  __shared__ int s_wn[8];
   const int R = R_dev ? *R_dev : R_max;
   const int r = blockIdx.x;
   if (r >= R) return;
@@ -221,6 +225,9 @@ __global__ void __launch_bounds__(256) expand_f32_kernel(const float* __restrict
   }
   __syncthreads();
   if (threadIdx.x < S) la_out[(long long)r * S + threadIdx.x] = la[threadIdx.x];
+  TopList best;
+  best.init();
+  float admit = -INFINITY;
   for (int k = threadIdx.x; k < V; k += blockDim.x) {
     float out = -INFINITY;
     if (k != blank) {
@@ -232,7 +239,40 @@ __global__ void __launch_bounds__(256) expand_f32_kernel(const float* __restrict
         out = mx + logf(s);
       }
     }
-    ldnb[(long long)r * V + k] = out;
+    if (ldnb) ldnb[(long long)r * V + k] = out;
+    if (cand.n && out > admit) {          // the blank column is -inf and never a candidate
+      best.insert(out, k);
+      admit = best.nth(cand.N);
+    }
+  }
+  if (cand.n == nullptr) return;
+  // ChooseNBestExpansions, first stage: this row's N best non-blank tokens
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int wn = warp_merge_lists(best, cand.N, s_wv[warp], s_wk[warp]);
+  if (lane == 0) s_wn[warp] = wn;
+  __syncthreads();
+  if (warp == 0) {
+    int pos = 0;
+    const int mine = lane < 8 ? s_wn[lane] : 0;
+    int cnt = 0;
+    for (int j = 0; j < cand.N; ++j) {
+      float bv = (pos < mine) ? s_wv[lane][pos] : -INFINITY;
+      int bk = (pos < mine) ? s_wk[lane][pos] : 0x7fffffff;
+      int bl = lane;
+#pragma unroll
+      for (int o = 4; o > 0; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+        const int ok = __shfl_xor_sync(0xffffffffu, bk, o);
+        const int ol = __shfl_xor_sync(0xffffffffu, bl, o);
+        if (cand_better(ov, ok, bv, bk)) { bv = ov; bk = ok; bl = ol; }
+      }
+      bv = __shfl_sync(0xffffffffu, bv, 0); bk = __shfl_sync(0xffffffffu, bk, 0); bl = __shfl_sync(0xffffffffu, bl, 0);
+      if (bv == -INFINITY) break;
+      if (lane == 0) { cand.v[(long long)r * kMaxBeam + j] = bv; cand.k[(long long)r * kMaxBeam + j] = bk; }
+      if (lane == bl) ++pos;
+      ++cnt;
+    }
+    if (lane == 0) cand.n[r] = cnt;
   }
 }
 
@@ -274,10 +314,10 @@ void launch_log_softmax(const JoinerRows& rows, int blank, float* z, cudaStream_
 
 void launch_expand_f32(const float* logp, const float* ld_old, const int* row_slen, const int* R_dev,
                        int R_max, int S, int V, int blank, float* ldphi, float* ldnb, float* la,
-                       double* ldphi_d, double* la_d, cudaStream_t st) {
+                       double* ldphi_d, double* la_d, const CandOut& cand, cudaStream_t st) {
   if (R_max <= 0) return;
   expand_f32_kernel<<<R_max, 256, 0, st>>>(logp, ld_old, row_slen, R_dev, R_max, S, V, blank, ldphi,
-                                           ldnb, la, ldphi_d, la_d);
+                                           ldnb, la, ldphi_d, la_d, cand);
 }
 
 void launch_rows_from_groups(const int* row_group, const int* seg_len, int R, int S, int* row_e0,

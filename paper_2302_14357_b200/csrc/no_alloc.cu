@@ -62,6 +62,6 @@ extern "C" int tw_joiner_expand_noalloc(const float* W_out, const float* b_out, 
   launch_joiner_f32(jr, W_out, b_out, logp, st);
   launch_log_softmax(jr, blank, logp, st);
   launch_expand_f32(logp, ld_old, row_slen, nullptr, R, S, V, blank, out_ldphi, out_ldnb, out_la, nullptr,
-                    nullptr, st);
+                    nullptr, CandOut{}, st);
   return cudaGetLastError() == cudaSuccess ? TW_OK : TW_ERR_CUDA;
 }

@@ -171,7 +171,7 @@ int build_workspace(tw_handle* h) {
   hs.stateless = (h->pred_kind == TW_PRED_STATELESS);
   const size_t nb = (size_t)B, nslot = nb * hs.capSlot, nB = nb * hs.capB, R = (size_t)h->R_max;
   int** per_utt[] = {&hs.len, &hs.t0, &hs.slen, &hs.nA, &hs.nB, &hs.nTop, &hs.iters, &hs.status,
-                     &hs.cursor, &hs.n_new, &hs.calls, &hs.joins, &hs.row_off};
+                     &hs.cursor, &hs.n_new, &hs.calls, &hs.joins, &hs.row_off, &hs.new_off};
   for (int** p : per_utt) TW_TRY(dev_alloc(h, p, nb));
   TW_TRY(dev_alloc(h, &hs.A_slot, nb * kMaxBeam));
   TW_TRY(dev_alloc(h, &hs.A_ls, nb * kMaxBeam));
@@ -202,6 +202,9 @@ int build_workspace(tw_handle* h) {
   TW_TRY(dev_alloc(h, &hs.ldphi, R));
   TW_TRY(dev_alloc(h, &hs.la, R * S));
   TW_TRY(dev_alloc(h, &hs.ldphi_d, R));
+  TW_TRY(dev_alloc(h, &hs.cand_v, R * kMaxBeam));
+  TW_TRY(dev_alloc(h, &hs.cand_k, R * kMaxBeam));
+  TW_TRY(dev_alloc(h, &hs.cand_n, R));
   TW_TRY(dev_alloc(h, &hs.la_d, R * S));
   TW_TRY(dev_alloc(h, &hs.ldnb, R * h->V));
   TW_TRY(dev_alloc(h, &hs.logp, R * S * h->V));
@@ -268,11 +271,11 @@ namespace tw {
 void enqueue_joiner_logits(tw_handle* h, const JoinerRows& rows, float* logp, cudaStream_t st, int* launches);
 void enqueue_joiner_expand_f32(tw_handle* h, const JoinerRows& rows, const float* ld_old, float* logp,
                                float* ldphi, float* ldnb, float* la, double* ldphi_d, double* la_d,
-                               cudaStream_t st, int* launches) {
+                               const CandOut& cand, cudaStream_t st, int* launches) {
   enqueue_joiner_logits(h, rows, logp, st, launches);
   launch_log_softmax(rows, h->blank, logp, st);
   launch_expand_f32(logp, ld_old, rows.row_slen, rows.R_dev, rows.R_max, rows.S, rows.V, h->blank, ldphi,
-                    ldnb, la, ldphi_d, la_d, st);
+                    ldnb, la, ldphi_d, la_d, cand, st);
   *launches += 2;
 }
 

@@ -54,6 +54,6 @@ namespace tw {
 // stages shared by tw_decode and the stage entry points
 void enqueue_joiner_expand_f32(tw_handle* h, const JoinerRows& rows, const float* ld_old, float* logp,
                                float* ldphi, float* ldnb, float* la, double* ldphi_d, double* la_d,
-                               cudaStream_t st, int* launches);
+                               const CandOut& cand, cudaStream_t st, int* launches);
 }
 

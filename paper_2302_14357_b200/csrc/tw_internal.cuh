@@ -66,10 +66,17 @@ void launch_joiner_f32(const JoinerRows& rows, const float* W_out, const float* 
                        cudaStream_t st);
 // in place: z[(r,t), :] -> log softmax; padding frames get (0 at blank, -inf elsewhere)
 void launch_log_softmax(const JoinerRows& rows, int blank, float* z, cudaStream_t st);
-// Eq. 3-7 from materialised log J
+// Per-row candidates of ChooseNBestExpansions: the row's best N non-blank tokens, best first
+// (score descending, then token ascending).  v, k are [R][kMaxBeam]; n[r] is how many are valid.
+struct CandOut {
+  float* v; int* k; int* n; int N;
+};
+// Eq. 3-7 from materialised log J; ldnb may be nullptr when only the candidates are wanted, and
+// cand.n may be nullptr when they are not
 void launch_expand_f32(const float* logp, const float* ld_old, const int* row_slen, const int* R_dev,
                        int R_max, int S, int V, int blank, float* ldphi, float* ldnb, float* la,
-                       double* ldphi_d, double* la_d, cudaStream_t st);   // float64 copies optional
+                       double* ldphi_d, double* la_d, const CandOut& cand,
+                       cudaStream_t st);   // float64 copies optional
 // helper for the stage entry points: row_e0[r] = row_group[r] * S, row_slen[r] = seg_len[row_group[r]]
 void launch_rows_from_groups(const int* row_group, const int* seg_len, int R, int S, int* row_e0,
                              int* row_slen, cudaStream_t st);
@@ -100,7 +107,7 @@ struct HypState {
   int *new_slot, *new_par, *new_tok;
   // compacted rows of the current step: [B*N]
   int *row_b, *row_e0, *row_p, *row_slen; float* row_ld;   // row_ld [R][S]
-  int *row_off;     // [B]
+  int *row_off, *new_off;     // [B] first row / first work-list entry of each utterance
   // compacted predictor work list: [B*N]
   int *pw_new, *pw_par, *pw_tok;
   int* scalars;           // [kScCount] device scalars
@@ -108,6 +115,7 @@ struct HypState {
   // stage outputs of the current step
   float *ldphi, *la, *ldnb, *logp;
   double *ldphi_d, *la_d;   // float64 copies of ldphi / la (nullptr: use the float32 ones)
+  float* cand_v; int* cand_k; int* cand_n;   // per-row expansion candidates [R][kMaxBeam], [R]
   // InitPredictor result (LSTM only): [L][2][Hd], [J]
   const float* init_hc; const float* init_Pp;
 };
