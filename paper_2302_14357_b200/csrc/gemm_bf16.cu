@@ -1,8 +1,10 @@
 // bf16 tensor-core GEMM for sm_100a:  C[m, n] = sum_k A[m, k] * B[n, k] (+ bias[n]), fp32 accumulate.
-// TMA (128-byte swizzle) feeds a multi-stage shared-memory ring; one thread issues tcgen05.mma into a
-// TMEM accumulator; four warps read the accumulator back with tcgen05.ld and write the tile.
-// Warp roles: 0 = TMA producer, 1 = MMA issuer and TMEM owner, 2..5 = epilogue (one TMEM lane quarter
-// each).  Every wait is bounded (sm100::mbar_wait); on a timeout the kernel raises *err and exits.
+// Persistent: one CTA per SM walks the tile list.  TMA (128-byte swizzle) feeds a multi-stage
+// shared-memory ring; one thread issues tcgen05.mma into one of two TMEM accumulator buffers, so the
+// epilogue of a tile (tcgen05.ld, bias, stores) overlaps the contraction of the next.
+// Warp roles: 0 = TMA producer, 1 = MMA issuer and TMEM owner, 2..9 = epilogue (two warps per TMEM
+// lane quarter, half of the columns each).  Every wait is bounded (sm100::mbar_wait); on a timeout
+// the kernel raises *err and every role leaves its loop.
 #include "bf16_path.cuh"
 #include "sm100.cuh"
 
@@ -13,6 +15,8 @@ namespace {
 using namespace sm100;
 
 constexpr int BM = 128, BK = 64;
+constexpr int kEpiWarps = 8;
+constexpr int kThreadsGemm = 64 + 32 * kEpiWarps;
 
 template <int BN>
 struct Cfg {
@@ -22,7 +26,7 @@ struct Cfg {
 };
 
 template <int BN>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(kThreadsGemm, 1)
 gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmBf16Params p) {
   using C = Cfg<BN>;
   extern __shared__ uint8_t smem_raw[];
@@ -31,12 +35,14 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   uint8_t* sB = smem + C::kStages * C::kABytes;
   uint64_t* full = reinterpret_cast<uint64_t*>(sB + C::kStages * C::kBBytes);
   uint64_t* empty = full + C::kStages;
-  uint64_t* accum = empty + C::kStages;
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(accum + 1);
+  uint64_t* acc_full = empty + C::kStages;     // [2]
+  uint64_t* acc_empty = acc_full + 2;          // [2]
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(acc_empty + 2);
 
   const int M = p.M_dev ? *p.M_dev : p.M;
-  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
-  if (m0 >= M) return;
+  const int m_tiles = (M + BM - 1) / BM, n_tiles = (p.N + BN - 1) / BN;
+  const int num_tiles = m_tiles * n_tiles;
+  if ((int)blockIdx.x >= num_tiles) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_kb = (p.K + BK - 1) / BK;
 
@@ -44,11 +50,11 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     prefetch_tensormap(&tmA);
     prefetch_tensormap(&tmB);
     for (int s = 0; s < C::kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    mbar_init(accum, 1);
+    for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], kEpiWarps); }
     fence_barrier_init();
     fence_proxy_async_smem();
   }
-  if (warp == 1) { tmem_alloc(tmem_holder, BN); tmem_relinquish(); }
+  if (warp == 1) { tmem_alloc(tmem_holder, 2 * BN); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -56,48 +62,71 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
   if (warp == 0) {
     if (lane == 0) {
-      for (int kb = 0; kb < num_kb; ++kb) {
-        const int s = kb % C::kStages;
-        const uint32_t ph = (kb / C::kStages) & 1;
-        if (!mbar_wait(&empty[s], ph ^ 1, p.err)) break;
-        mbar_expect_tx(&full[s], C::kABytes + C::kBBytes);
-        tma_load_2d(sA + s * C::kABytes, &tmA, &full[s], kb * BK, m0);
-        tma_load_2d(sB + s * C::kBBytes, &tmB, &full[s], kb * BK, n0);
+      uint32_t it = 0;                       // k-block counter across tiles: the ring never restarts
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        const int m0 = (tile / n_tiles) * BM, n0 = (tile % n_tiles) * BN;
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+          const int s = it % C::kStages;
+          const uint32_t ph = (it / C::kStages) & 1;
+          ok = mbar_wait(&empty[s], ph ^ 1, p.err);
+          if (!ok) break;
+          mbar_expect_tx(&full[s], C::kABytes + C::kBBytes);
+          tma_load_2d(sA + s * C::kABytes, &tmA, &full[s], kb * BK, m0);
+          tma_load_2d(sB + s * C::kBBytes, &tmB, &full[s], kb * BK, n0);
+        }
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
       constexpr uint32_t idesc = make_idesc_bf16(BM, BN);
+      uint32_t it = 0, lt = 0;               // lt: tiles done by this CTA
       bool ok = true;
-      for (int kb = 0; kb < num_kb && ok; ++kb) {
-        const int s = kb % C::kStages;
-        const uint32_t ph = (kb / C::kStages) & 1;
-        ok = mbar_wait(&full[s], ph, p.err);
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++lt) {
+        const uint32_t buf = lt & 1, aph = (lt >> 1) & 1;
+        ok = mbar_wait(&acc_empty[buf], aph ^ 1, p.err);      // epilogue has drained this buffer
         if (!ok) break;
         tc_fence_after();
-        const uint32_t a_addr = smem_u32(sA + s * C::kABytes), b_addr = smem_u32(sB + s * C::kBBytes);
+        const uint32_t tmem_d = tmem_base + buf * BN;
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+          const int s = it % C::kStages;
+          const uint32_t ph = (it / C::kStages) & 1;
+          ok = mbar_wait(&full[s], ph, p.err);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t a_addr = smem_u32(sA + s * C::kABytes), b_addr = smem_u32(sB + s * C::kBBytes);
 #pragma unroll
-        for (int k = 0; k < BK / 16; ++k)
-          umma_bf16(tmem_base, make_desc_k_sw128(a_addr + k * 32), make_desc_k_sw128(b_addr + k * 32), idesc,
-                    (kb | k) != 0);
-        umma_commit(&empty[s]);
+          for (int k = 0; k < BK / 16; ++k)
+            umma_bf16(tmem_d, make_desc_k_sw128(a_addr + k * 32), make_desc_k_sw128(b_addr + k * 32), idesc,
+                      (kb | k) != 0);
+          umma_commit(&empty[s]);
+        }
+        if (ok) umma_commit(&acc_full[buf]);
       }
-      umma_commit(accum);
     }
   } else {
-    const int q = warp & 3;
-    const int m = m0 + q * 32 + lane;
-    bool ok = mbar_wait(accum, 0, p.err);
-    ok = __all_sync(0xffffffffu, ok);
-    tc_fence_after();
-    if (ok) {
+    const int ew = warp - 2;                 // 0..7
+    const int q = warp & 3;                  // TMEM lane quarter this warp may read
+    const int half = ew >> 2;                // which half of the tile's columns
+    constexpr int kColsPerWarp = BN / 2;
+    uint32_t lt = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++lt) {
+      const int m0 = (tile / n_tiles) * BM, n0 = (tile % n_tiles) * BN;
+      const uint32_t buf = lt & 1, aph = (lt >> 1) & 1;
+      ok = mbar_wait(&acc_full[buf], aph, p.err);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const int m = m0 + q * 32 + lane;
       float* crow = nullptr;
       if (m < M) crow = p.C + (long long)(p.oidx ? p.oidx[m] : m) * p.ldC;
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
+      for (int c = 0; c < kColsPerWarp / 32; ++c) {
         float v[32];
-        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), v);
-        const int nb = n0 + c * 32;
+        const int col = half * kColsPerWarp + c * 32;
+        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + buf * BN + (uint32_t)col, v);
+        const int nb = n0 + col;
         if (crow != nullptr && nb < p.N) {
           if (nb + 32 <= p.N && ((reinterpret_cast<uintptr_t>(crow + nb) & 15) == 0)) {
 #pragma unroll
@@ -115,11 +144,15 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           }
         }
       }
+      // all of this warp's TMEM reads have completed (tmem_ld32 waits): hand the buffer back
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&acc_empty[buf]);
     }
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) tmem_dealloc(tmem_base, BN);
+  if (warp == 1) tmem_dealloc(tmem_base, 2 * BN);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -162,15 +195,22 @@ int gemm_bf16_setup() {
 void launch_gemm_bf16(const CUtensorMap& tmA, const CUtensorMap& tmB128, const CUtensorMap& tmB256,
                       const GemmBf16Params& p, cudaStream_t st) {
   if (p.M <= 0 || p.N <= 0) return;
+  static int num_sms = 0;
+  if (num_sms == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms <= 0) num_sms = 148;
+  }
   const int mt = (p.M + BM - 1) / BM;
-  const int nt256 = (p.N + 255) / 256;
+  const int nt256 = (p.N + 255) / 256, nt128 = (p.N + 127) / 128;
   // small problems: narrower tiles put more SMs to work
-  if ((long long)mt * nt256 >= 148) {
-    dim3 grid(nt256, mt);
-    gemm_bf16_kernel<256><<<grid, 192, Cfg<256>::kSmem, st>>>(tmA, tmB256, p);
+  if ((long long)mt * nt256 >= num_sms) {
+    const int grid = (int)((long long)mt * nt256 < num_sms ? mt * nt256 : num_sms);
+    gemm_bf16_kernel<256><<<grid, kThreadsGemm, Cfg<256>::kSmem, st>>>(tmA, tmB256, p);
   } else {
-    dim3 grid((p.N + 127) / 128, mt);
-    gemm_bf16_kernel<128><<<grid, 192, Cfg<128>::kSmem, st>>>(tmA, tmB128, p);
+    const long long tiles = (long long)mt * nt128;
+    const int grid = (int)(tiles < num_sms ? tiles : num_sms);
+    gemm_bf16_kernel<128><<<grid, kThreadsGemm, Cfg<128>::kSmem, st>>>(tmA, tmB128, p);
   }
 }
 

@@ -272,7 +272,9 @@ __global__ void __launch_bounds__(kStepThreads) hyp_step_kernel(HypState hs) {
       double v = -INFINITY;
       if (t < slen && hs.logp != nullptr) {
         const double a = hs.la_d ? hs.la_d[r * S + t] : (double)hs.la[r * S + t];
-        v = s_Als[h] + a + (double)hs.logp[(r * S + t) * V + k];
+        double lj = (double)hs.logp[(r * S + t) * V + k];
+        if (hs.lse) lj -= (double)hs.lse[r * S + t];
+        v = s_Als[h] + a + lj;
       }
       hs.A_ld[((long long)b * kMaxBeam + i) * S + t] = v;
     }

@@ -201,6 +201,10 @@ int build_workspace(tw_handle* h) {
   TW_TRY(dev_alloc(h, &hs.rows_total, (size_t)2));
   TW_TRY(dev_alloc(h, &hs.ldphi, R));
   TW_TRY(dev_alloc(h, &hs.la, R * S));
+  if (scan_select_fits(S, h->V)) {
+    TW_TRY(scan_select_setup());
+    TW_TRY(dev_alloc(h, &hs.lse, R * S));
+  }
   TW_TRY(dev_alloc(h, &hs.ldphi_d, R));
   TW_TRY(dev_alloc(h, &hs.cand_v, R * kMaxBeam));
   TW_TRY(dev_alloc(h, &hs.cand_k, R * kMaxBeam));
@@ -269,14 +273,31 @@ int init_impl(tw_handle* h, const tw_model* m, const tw_config* c) {
 
 namespace tw {
 void enqueue_joiner_logits(tw_handle* h, const JoinerRows& rows, float* logp, cudaStream_t st, int* launches);
+void enqueue_scan(tw_handle* h, const JoinerRows& rows, const float* ld_old, float* logp, float* ldphi,
+                  float* ldnb, float* la, double* ldphi_d, double* la_d, const CandOut& cand, cudaStream_t st,
+                  int* launches);
 void enqueue_joiner_expand_f32(tw_handle* h, const JoinerRows& rows, const float* ld_old, float* logp,
                                float* ldphi, float* ldnb, float* la, double* ldphi_d, double* la_d,
                                const CandOut& cand, cudaStream_t st, int* launches) {
   enqueue_joiner_logits(h, rows, logp, st, launches);
-  launch_log_softmax(rows, h->blank, logp, st);
-  launch_expand_f32(logp, ld_old, rows.row_slen, rows.R_dev, rows.R_max, rows.S, rows.V, h->blank, ldphi,
-                    ldnb, la, ldphi_d, la_d, cand, st);
-  *launches += 2;
+  enqueue_scan(h, rows, ld_old, logp, ldphi, ldnb, la, ldphi_d, la_d, cand, st, launches);
+}
+
+// softmax, Eq. 3-7 and the rows' candidates from the raw logits in `logp`
+void enqueue_scan(tw_handle* h, const JoinerRows& rows, const float* ld_old, float* logp, float* ldphi,
+                  float* ldnb, float* la, double* ldphi_d, double* la_d, const CandOut& cand, cudaStream_t st,
+                  int* launches) {
+  if (h->hs.lse != nullptr) {
+    ScanSelectArgs a{logp, ld_old, rows.row_slen, rows.R_dev, rows.R_max, rows.S, rows.V, h->blank,
+                     h->hs.lse, ldphi, ldnb, la, ldphi_d, la_d, cand};
+    launch_scan_select(a, st);
+    *launches += 1;
+  } else {
+    launch_log_softmax(rows, h->blank, logp, st);
+    launch_expand_f32(logp, ld_old, rows.row_slen, rows.R_dev, rows.R_max, rows.S, rows.V, h->blank, ldphi,
+                      ldnb, la, ldphi_d, la_d, cand, st);
+    *launches += 2;
+  }
 }
 
 // z[(r, t), :] = W_out tanh(E + Pp) + b_out into `logp` (rows of padding frames hold no result)

@@ -52,6 +52,10 @@ struct tw_handle {
 
 namespace tw {
 // stages shared by tw_decode and the stage entry points
+void enqueue_joiner_logits(tw_handle* h, const JoinerRows& rows, float* logp, cudaStream_t st, int* launches);
+void enqueue_scan(tw_handle* h, const JoinerRows& rows, const float* ld_old, float* logp, float* ldphi,
+                  float* ldnb, float* la, double* ldphi_d, double* la_d, const CandOut& cand, cudaStream_t st,
+                  int* launches);
 void enqueue_joiner_expand_f32(tw_handle* h, const JoinerRows& rows, const float* ld_old, float* logp,
                                float* ldphi, float* ldnb, float* la, double* ldphi_d, double* la_d,
                                const CandOut& cand, cudaStream_t st, int* launches);

@@ -77,6 +77,18 @@ void launch_expand_f32(const float* logp, const float* ld_old, const int* row_sl
                        int R_max, int S, int V, int blank, float* ldphi, float* ldnb, float* la,
                        double* ldphi_d, double* la_d, const CandOut& cand,
                        cudaStream_t st);   // float64 copies optional
+// Softmax + Eq. 3-7 + per-row candidates from RAW logits z [R, S, V] read once into shared memory
+// (scan_select.cu).  Every output pointer is optional.
+struct ScanSelectArgs {
+  const float* z; const float* ld_old; const int* row_slen; const int* R_dev;
+  int R_max, S, V, blank;
+  float* lse_out;      // [R, S] softmax normalisers: log J(t, k) = z[t, k] - lse[t]
+  float *ldphi, *ldnb, *la; double *ldphi_d, *la_d;
+  CandOut cand;
+};
+bool scan_select_fits(int S, int V);   // the row's S x V logits fit in shared memory
+int scan_select_setup();
+void launch_scan_select(const ScanSelectArgs& a, cudaStream_t st);
 // helper for the stage entry points: row_e0[r] = row_group[r] * S, row_slen[r] = seg_len[row_group[r]]
 void launch_rows_from_groups(const int* row_group, const int* seg_len, int R, int S, int* row_e0,
                              int* row_slen, cudaStream_t st);
@@ -114,6 +126,7 @@ struct HypState {
   long long* rows_total;  // [2]: sum over steps of rows R, and of rows x their segment's frames
   // stage outputs of the current step
   float *ldphi, *la, *ldnb, *logp;
+  float* lse;   // [R][S]; when set, logp holds raw logits and log J = logp - lse
   double *ldphi_d, *la_d;   // float64 copies of ldphi / la (nullptr: use the float32 ones)
   float* cand_v; int* cand_k; int* cand_n;   // per-row expansion candidates [R][kMaxBeam], [R]
   // InitPredictor result (LSTM only): [L][2][Hd], [J]

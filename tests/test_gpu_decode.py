@@ -9,10 +9,12 @@ from helpers import SCORE_TOL, check_against_oracle, nbest_from_arrays, oracle_m
 pytestmark = pytest.mark.gpu
 
 
-def _run(cfg, S, N=None, batch=None, T=None, lengths=None, max_iters=0, mode=0, check=None):
+def _run(cfg, S, N=None, batch=None, T=None, lengths=None, max_iters=0, mode=0, check=None, mutate=None):
     from paper_2302_14357_b200.binding import TwDecoder, weights_from_synth
     N = N or cfg.N
     m = tw_synth.make_model(cfg)
+    if mutate is not None:
+        mutate(m)
     enc, lens = tw_synth.make_encoder_batch(cfg, batch)
     if T is not None:
         enc = np.ascontiguousarray(enc[:, :T])
@@ -78,6 +80,16 @@ def test_many_merges_small_vocab():
     """V=3: few distinct sequences, so AddAndMerge fires constantly."""
     cfg = _tiny("lstm", 1, V=3, seed=12).with_(blank_bias=0.0)
     _run(cfg, 3, N=2, lengths=[23, 11, 23, 8, 2, 23])
+
+
+def test_uniform_joiner_exact_ties():
+    """W_out = 0: every token of a row has the same score, so the selection runs on ties alone
+    (smaller hypothesis index, then smaller token) and more tokens tie than the fast path holds."""
+    def flat(m):
+        m.W_out[:] = 0.0
+        m.b_out[:] = 0.0
+    cfg = _tiny("stateless", V=300, seed=3)
+    _run(cfg, 3, N=4, lengths=[7, 3, 6, 1, 2, 5], mutate=flat, max_iters=3)
 
 
 @pytest.mark.parametrize("S", [1, 2, 3, 5])

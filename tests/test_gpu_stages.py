@@ -128,7 +128,34 @@ def test_joiner_expand_is_the_composition():
     a = dec.expand(logp, ld_old, seg_len[row_group])
     b = dec.joiner_expand(E, Pp, row_group, seg_len, ld_old)
     for x, y in zip(a, b):
-        _allclose_inf(x.cpu().numpy(), y.cpu().numpy(), 1e-6)
+        _allclose_inf(x.cpu().numpy(), y.cpu().numpy(), 1e-5)
+
+
+@pytest.mark.parametrize("S,V", [(1, 70), (3, 1000), (10, 257), (50, 130)])
+def test_joiner_expand_matches_oracle_chain(S, V):
+    """The one-call stage against joiner -> softmax -> Eq. 3-7 of the oracle, ragged segments."""
+    cfg = _small_cfg(V=V)
+    m, dec = _decoder(cfg, S)
+    om = oracle_model(m)
+    rng = np.random.default_rng(S * 7 + V)
+    G, R = 3, 6
+    enc = rng.standard_normal((G, S, cfg.D_enc)).astype(np.float32)
+    pred = rng.standard_normal((R, cfg.P)).astype(np.float32)
+    row_group = np.array([0, 1, 2, 2, 1, 0], np.int32)
+    seg_len = np.array([S, max(1, S // 2), max(1, S - 1)], np.int32)
+    ld_old = (rng.standard_normal((R, S)) - 2).astype(np.float32)
+    ld_old[0, 1:] = -np.inf
+    E = dec.project_encoder(enc).reshape(G, S, cfg.J)
+    Pp = (pred.astype(np.float64) @ om.W_p.T).astype(np.float32)
+    ldphi, ldnb, la = [x.cpu().numpy() for x in dec.joiner_expand(E, Pp, row_group, seg_len, ld_old)]
+    for r in range(R):
+        sl = seg_len[row_group[r]]
+        lj = rm.joiner_log_probs(om, enc[row_group[r], :sl], pred[r:r + 1])
+        lo = ld_old[r:r + 1, :sl].astype(np.float64)
+        lBl = sm.blank_product(lj)
+        ld = sm.nonblank_expansion_t(lj, lBl, lo)
+        _allclose_inf(ldnb[r], sm.nonblank_expansion(ld)[0], 2 * STAGE_TOL)
+        _allclose_inf(ldphi[r:r + 1], sm.blank_expansion(lBl, lo), 2 * STAGE_TOL)
 
 
 @pytest.mark.parametrize("pred,layers", [("stateless", 0), ("lstm", 1), ("lstm", 2)])
