@@ -15,6 +15,9 @@ struct GemmBf16Params {
   long long ldC;
   const float* bias;  // optional [N]
   int* err;           // device error word, raised by a wait that gave up
+  const float* addend = nullptr;   // optional: row m also gets addend[(add_idx ? add_idx[m] : m) * ld_add + n]
+  const int* add_idx = nullptr;
+  long long ld_add = 0;
 };
 
 // 2-D bf16 tensor map over a row-major [rows, K] matrix, box = 64 x box_rows, 128-byte swizzle.

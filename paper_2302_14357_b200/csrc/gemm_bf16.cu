@@ -120,7 +120,11 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       tc_fence_after();
       const int m = m0 + q * 32 + lane;
       float* crow = nullptr;
-      if (m < M) crow = p.C + (long long)(p.oidx ? p.oidx[m] : m) * p.ldC;
+      const float* arow = nullptr;           // optional per-row addend (gathered)
+      if (m < M) {
+        crow = p.C + (long long)(p.oidx ? p.oidx[m] : m) * p.ldC;
+        if (p.addend) arow = p.addend + (long long)(p.add_idx ? p.add_idx[m] : m) * p.ld_add;
+      }
 #pragma unroll 1
       for (int c = 0; c < kColsPerWarp / 32; ++c) {
         float v[32];
@@ -129,18 +133,20 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const int nb = n0 + col;
         if (crow != nullptr && nb < p.N) {
           if (nb + 32 <= p.N && ((reinterpret_cast<uintptr_t>(crow + nb) & 15) == 0)) {
+            if (p.bias) {
 #pragma unroll
-            for (int j = 0; j < 32; j += 4) {
-              float4 o;
-              o.x = v[j] + (p.bias ? p.bias[nb + j] : 0.f);
-              o.y = v[j + 1] + (p.bias ? p.bias[nb + j + 1] : 0.f);
-              o.z = v[j + 2] + (p.bias ? p.bias[nb + j + 2] : 0.f);
-              o.w = v[j + 3] + (p.bias ? p.bias[nb + j + 3] : 0.f);
-              *reinterpret_cast<float4*>(crow + nb + j) = o;
+              for (int j = 0; j < 32; ++j) v[j] += p.bias[nb + j];
             }
+            if (arow) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) v[j] += arow[nb + j];
+            }
+#pragma unroll
+            for (int j = 0; j < 32; j += 4)
+              *reinterpret_cast<float4*>(crow + nb + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
           } else {
             for (int j = 0; j < 32; ++j)
-              if (nb + j < p.N) crow[nb + j] = v[j] + (p.bias ? p.bias[nb + j] : 0.f);
+              if (nb + j < p.N) crow[nb + j] = v[j] + (p.bias ? p.bias[nb + j] : 0.f) + (arow ? arow[nb + j] : 0.f);
           }
         }
       }

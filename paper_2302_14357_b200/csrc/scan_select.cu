@@ -13,8 +13,8 @@ namespace tw {
 
 namespace {
 
-constexpr int kT = 256;
-constexpr int kGroups = 16;        // 16 groups of 16 threads: their maxima bound the N-th best value
+constexpr int kMaxT = 1024;         // threads per CTA: 256 for small rows, 1024 when one CTA fills the SM
+constexpr int kMaxGroups = kMaxT / 16;   // groups of 16 threads: their maxima bound the N-th best value
 constexpr int kSurvCap = 192;
 
 __device__ __forceinline__ float wmax(float v) {
@@ -28,17 +28,24 @@ __device__ __forceinline__ float wsum(float v) {
   return v;
 }
 
-__global__ void __launch_bounds__(kT) scan_select_kernel(ScanSelectArgs a) {
+template <bool FAST>
+__device__ __forceinline__ float ex(float x) { return FAST ? __expf(x) : expf(x); }
+template <bool FAST>
+__device__ __forceinline__ float lg(float x) { return FAST ? __logf(x) : logf(x); }
+
+// FAST: hardware exp2/log2 approximations (bf16 mode, where the operands carry 2^-9 already)
+template <bool FAST>
+__global__ void __launch_bounds__(kMaxT) scan_select_kernel(ScanSelectArgs a) {
   extern __shared__ __align__(16) float zs[];          // [S][V] logits of this row; row 0 later holds dnb
   __shared__ float s_lse[kMaxSeg], s_w[kMaxSeg];
-  __shared__ float s_gmax[kGroups];
+  __shared__ float s_gmax[kMaxGroups];
   __shared__ float s_bound;
   __shared__ int s_nsurv;
   __shared__ float s_sv[kSurvCap];
   __shared__ int s_sk[kSurvCap];
-  __shared__ float s_wv[kT / 32][kMaxBeam];
-  __shared__ int s_wk[kT / 32][kMaxBeam];
-  __shared__ int s_wn[kT / 32];
+  __shared__ float s_wv[kMaxT / 32][kMaxBeam];
+  __shared__ int s_wk[kMaxT / 32][kMaxBeam];
+  __shared__ int s_wn[kMaxT / 32];
 
   const int R = a.R_dev ? *a.R_dev : a.R_max;
   const int r = blockIdx.x;
@@ -46,6 +53,7 @@ __global__ void __launch_bounds__(kT) scan_select_kernel(ScanSelectArgs a) {
   const int S = a.S, V = a.V, blank = a.blank;
   const int sl = a.row_slen ? a.row_slen[r] : S;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int kT = blockDim.x, nwarps = kT >> 5, ngroups = kT >> 4;
   const float* z = a.z + (long long)r * S * V;
 
   // ---- the one pass over global memory
@@ -61,16 +69,16 @@ __global__ void __launch_bounds__(kT) scan_select_kernel(ScanSelectArgs a) {
   __syncthreads();
 
   // ---- per-frame log-sum-exp: one warp per frame
-  for (int t = warp; t < sl; t += kT / 32) {
+  for (int t = warp; t < sl; t += nwarps) {
     const float* row = zs + t * V;
     float mx = -INFINITY;
     for (int k = lane; k < V; k += 32) mx = fmaxf(mx, row[k]);
     mx = wmax(mx);
     float s = 0.f;
-    for (int k = lane; k < V; k += 32) s += expf(row[k] - mx);
+    for (int k = lane; k < V; k += 32) s += ex<FAST>(row[k] - mx);
     s = wsum(s);
     if (lane == 0) {
-      const float lse = mx + logf(s);
+      const float lse = mx + lg<FAST>(s);
       s_lse[t] = lse;
       if (a.lse_out) a.lse_out[(long long)r * S + t] = lse;
     }
@@ -108,8 +116,8 @@ __global__ void __launch_bounds__(kT) scan_select_kernel(ScanSelectArgs a) {
       for (int t = 0; t < sl; ++t) mx = fmaxf(mx, s_w[t] + zs[t * V + k]);
       if (mx > -INFINITY) {
         float s = 0.f;
-        for (int t = 0; t < sl; ++t) s += expf(s_w[t] + zs[t * V + k] - mx);
-        out = mx + logf(s);
+        for (int t = 0; t < sl; ++t) s += ex<FAST>(s_w[t] + zs[t * V + k] - mx);
+        out = mx + lg<FAST>(s);
       }
     }
     if (sl > 0) zs[k] = out;                 // only this thread ever touches column k
@@ -126,13 +134,15 @@ __global__ void __launch_bounds__(kT) scan_select_kernel(ScanSelectArgs a) {
   if ((tid & 15) == 0) s_gmax[tid >> 4] = tmax;
   __syncthreads();
   if (warp == 0) {
-    const float mine = lane < kGroups ? s_gmax[lane] : -INFINITY;
-    int rank = 0;
-    for (int j = 0; j < kGroups; ++j) {
-      const float o = __shfl_sync(0xffffffffu, mine, j);
-      rank += (o > mine) || (o == mine && j < lane);
+    for (int g = lane; g < ngroups; g += 32) {
+      const float mine = s_gmax[g];
+      int rank = 0;
+      for (int j = 0; j < ngroups; ++j) {
+        const float o = s_gmax[j];
+        rank += (o > mine) || (o == mine && j < g);
+      }
+      if (rank == N - 1) s_bound = mine;       // N <= 16 <= ngroups: exactly one group has this rank
     }
-    if (lane < kGroups && rank == min(N, kGroups) - 1) s_bound = (N <= kGroups) ? mine : -INFINITY;
   }
   __syncthreads();
   const float bound = s_bound;
@@ -173,13 +183,13 @@ __global__ void __launch_bounds__(kT) scan_select_kernel(ScanSelectArgs a) {
   __syncthreads();
   if (warp == 0) {
     int pos = 0, cnt = 0;
-    const int mine = lane < kT / 32 ? s_wn[lane] : 0;
+    const int mine = lane < nwarps ? s_wn[lane] : 0;
     for (int j = 0; j < N; ++j) {
-      float bv = (pos < mine) ? s_wv[lane & 7][pos] : -INFINITY;
-      int bk = (pos < mine) ? s_wk[lane & 7][pos] : 0x7fffffff;
+      float bv = (pos < mine) ? s_wv[lane][pos] : -INFINITY;
+      int bk = (pos < mine) ? s_wk[lane][pos] : 0x7fffffff;
       int bl = lane;
 #pragma unroll
-      for (int o = 4; o > 0; o >>= 1) {
+      for (int o = 16; o > 0; o >>= 1) {
         const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
         const int ok = __shfl_xor_sync(0xffffffffu, bk, o);
         const int ol = __shfl_xor_sync(0xffffffffu, bl, o);
@@ -202,13 +212,18 @@ size_t scan_select_smem_bytes(int S, int V) { return (size_t)S * V * sizeof(floa
 bool scan_select_fits(int S, int V) { return scan_select_smem_bytes(S, V) <= (size_t)200 * 1024; }
 
 int scan_select_setup() {
-  return cudaFuncSetAttribute(scan_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) == cudaSuccess
-             ? TW_OK : TW_ERR_CUDA;
+  cudaError_t e1 = cudaFuncSetAttribute(scan_select_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  cudaError_t e2 = cudaFuncSetAttribute(scan_select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  return (e1 == cudaSuccess && e2 == cudaSuccess) ? TW_OK : TW_ERR_CUDA;
 }
 
-void launch_scan_select(const ScanSelectArgs& a, cudaStream_t st) {
+void launch_scan_select(const ScanSelectArgs& a, bool fast_math, cudaStream_t st) {
   if (a.R_max <= 0) return;
-  scan_select_kernel<<<a.R_max, kT, scan_select_smem_bytes(a.S, a.V), st>>>(a);
+  const size_t smem = scan_select_smem_bytes(a.S, a.V);
+  // a row that takes most of an SM's shared memory runs alone there: give it the whole SM's threads
+  const int threads = smem > 96 * 1024 ? 1024 : (smem > 48 * 1024 ? 512 : 256);
+  if (fast_math) scan_select_kernel<true><<<a.R_max, threads, smem, st>>>(a);
+  else scan_select_kernel<false><<<a.R_max, threads, smem, st>>>(a);
 }
 
 }  // namespace tw

@@ -52,8 +52,10 @@ int make_bf16_mat(tw_handle* h, Bf16Mat* m, const float* src, long long rows, lo
 }
 
 void gemm_bf16(tw_handle* h, const Bf16Mat& A, const Bf16Mat& B, const int* M_dev, int M, float* C, const int* oidx,
-               long long ldC, const float* bias, cudaStream_t st) {
+               long long ldC, const float* bias, cudaStream_t st, const float* addend = nullptr,
+               const int* add_idx = nullptr, long long ld_add = 0) {
   GemmBf16Params p{M_dev, M, (int)B.rows, (int)A.K, C, oidx, ldC, bias, h->bf.err};
+  p.addend = addend; p.add_idx = add_idx; p.ld_add = ld_add;
   launch_gemm_bf16(A.as_A, B.as_B128, B.as_B256, p, st);
 }
 
@@ -79,7 +81,13 @@ void enqueue_predictor(tw_handle* h, const int* tok, const float* hc_in, const i
     const long long xld = (l == 0) ? h->emb_dim : stride;
     const int xk = (l == 0) ? h->emb_dim : Hd;
     const float* hp = hc_in + (long long)l * 2 * Hd;
-    if (h->mode == TW_MODE_BF16) {
+    if (h->mode == TW_MODE_BF16 && l == 0) {
+      // the input half W_ih[0] emb[tok] + b[0] is a table row; only W_hh[0] h_parent is contracted
+      launch_gather_concat_bf16(hp, idx_in, stride, Hd, nullptr, nullptr, 0, 0, n_dev, n_max, h->bf.X[0].ptr, st);
+      gemm_bf16(h, h->bf.X[0], h->bf.W_cat[0], n_dev, n_max, h->gates, nullptr, 4 * Hd, nullptr, st, h->bf.EmbProj,
+                tok, 4 * Hd);
+      *launches += 1;
+    } else if (h->mode == TW_MODE_BF16) {
       launch_gather_concat_bf16(x, xi, xld, xk, hp, idx_in, stride, Hd, n_dev, n_max, h->bf.X[l].ptr, st);
       gemm_bf16(h, h->bf.X[l], h->bf.W_cat[l], n_dev, n_max, h->gates, nullptr, 4 * Hd, h->b_l[l], st);
       *launches += 1;
@@ -148,12 +156,21 @@ int build_bf16(tw_handle* h) {
   if (h->pred_kind == TW_PRED_LSTM) {
     TW_TRY(make_bf16_mat(h, &h->bf.W_p, h->W_p, h->J, h->P, false, true));
     TW_TRY(make_bf16_mat(h, &h->bf.Htop, nullptr, h->R_max, h->Hd, true, false));
-    for (int l = 0; l < h->L; ++l) {
-      const int in = (l == 0) ? h->emb_dim : h->Hd;
-      TW_TRY(make_bf16_mat(h, &h->bf.W_cat[l], nullptr, 4 * h->Hd, in + h->Hd, false, true));
-      launch_gather_concat_bf16(h->W_ih[l], nullptr, in, in, h->W_hh[l], nullptr, h->Hd, h->Hd, nullptr, 4 * h->Hd,
+    {
+      // EmbProj[k] = W_ih[0] emb[k] + b[0]  (fp32 products of the stored weights, exact inputs)
+      TW_TRY(dev_alloc(h, &h->bf.EmbProj, (size_t)h->V * 4 * h->Hd));
+      GemmOperand a{h->emb, nullptr, h->emb_dim, h->W_ih[0], h->emb_dim, h->emb_dim};
+      GemmOperand none{};
+      GemmOut o{h->bf.EmbProj, nullptr, 4 * h->Hd, h->b_l[0]};
+      launch_gemm_f32(a, none, o, nullptr, h->V, 4 * h->Hd, 0);
+      TW_TRY(make_bf16_mat(h, &h->bf.W_cat[0], h->W_hh[0], 4 * h->Hd, h->Hd, false, true));
+      TW_TRY(make_bf16_mat(h, &h->bf.X[0], nullptr, h->R_max, h->Hd, true, false));
+    }
+    for (int l = 1; l < h->L; ++l) {
+      TW_TRY(make_bf16_mat(h, &h->bf.W_cat[l], nullptr, 4 * h->Hd, 2 * h->Hd, false, true));
+      launch_gather_concat_bf16(h->W_ih[l], nullptr, h->Hd, h->Hd, h->W_hh[l], nullptr, h->Hd, h->Hd, nullptr, 4 * h->Hd,
                                 h->bf.W_cat[l].ptr, 0);
-      TW_TRY(make_bf16_mat(h, &h->bf.X[l], nullptr, h->R_max, in + h->Hd, true, false));
+      TW_TRY(make_bf16_mat(h, &h->bf.X[l], nullptr, h->R_max, 2 * h->Hd, true, false));
     }
   }
   TW_CUDA(h, cudaGetLastError());
@@ -290,7 +307,7 @@ void enqueue_scan(tw_handle* h, const JoinerRows& rows, const float* ld_old, flo
   if (h->hs.lse != nullptr) {
     ScanSelectArgs a{logp, ld_old, rows.row_slen, rows.R_dev, rows.R_max, rows.S, rows.V, h->blank,
                      h->hs.lse, ldphi, ldnb, la, ldphi_d, la_d, cand};
-    launch_scan_select(a, st);
+    launch_scan_select(a, h->mode == TW_MODE_BF16, st);
     *launches += 1;
   } else {
     launch_log_softmax(rows, h->blank, logp, st);

@@ -26,11 +26,12 @@ struct tw_handle {
 
   // TW_MODE_BF16: bf16 copies of the GEMM operands with their tensor maps
   struct {
-    tw::Bf16Mat W_e, W_out, W_p, W_cat[tw::kMaxLayers];   // W_cat[l] = [W_ih[l] | W_hh[l]]  [4Hd, in+Hd]
+    tw::Bf16Mat W_e, W_out, W_p, W_cat[tw::kMaxLayers];   // W_cat[0] = W_hh[0] [4Hd, Hd]; W_cat[l>0] = [W_ih[l] | W_hh[l]] [4Hd, 2Hd]
     tw::Bf16Mat enc;                                      // [max_batch * max_T, D_enc]
     tw::Bf16Mat A_join;                                   // [R_max * S, J]  tanh(E + Pp)
-    tw::Bf16Mat X[tw::kMaxLayers];                        // [R_max, in+Hd]  LSTM layer inputs
+    tw::Bf16Mat X[tw::kMaxLayers];                        // LSTM layer inputs: [R_max, Hd] (layer 0: parent h) or [R_max, 2Hd]
     tw::Bf16Mat Htop;                                     // [R_max, Hd]
+    float* EmbProj = nullptr;   // [V, 4Hd] = emb W_ih[0]^T + b[0]: layer 0's input half, one row per token
     int* err = nullptr;                                   // device error word of the bounded waits
   } bf;
 
