@@ -1,0 +1,56 @@
+"""Full-size workloads in the launch configuration bench.py times (whole batch on the device), checked
+on sampled utterances the oracle can afford: fp32 mode exactly (near-tie protocol), bf16 mode by top-1."""
+import numpy as np
+import pytest
+
+import tw_synth
+from helpers import check_against_oracle, nbest_from_arrays, oracle_model
+from oracle import token_wise_search as tws
+
+pytestmark = pytest.mark.gpu
+
+
+def _decode(cfg, S, mode, T=None):
+    from paper_2302_14357_b200.binding import TwDecoder, weights_from_synth
+    m = tw_synth.make_model(cfg)
+    enc, lens = tw_synth.make_encoder_batch(cfg)
+    if T is not None:
+        enc, lens = np.ascontiguousarray(enc[:, :T]), np.minimum(lens, T)
+    dec = TwDecoder(weights_from_synth(m), N=cfg.N, S=S, mode=mode, max_batch=cfg.batch, max_T=enc.shape[1])
+    out = [x.cpu().numpy() for x in dec.decode(enc, lens)[:4]]
+    st = dec.stats()
+    dec.close()
+    return m, enc, lens, out, st
+
+
+@pytest.mark.parametrize("name,S,sample,T", [("c2", 3, (0, 37), None), ("c1", 5, (3, 30), None), ("c3", 3, (5, 90), 240)])
+def test_full_batch_fp32_sampled_utterances(name, S, sample, T):
+    cfg = tw_synth.get_config(name)
+    m, enc, lens, (tokens, olens, scores, status), st = _decode(cfg, S, 0, T)
+    assert st["limit_hits"] == 0 and np.all(status == 0)
+    # properties that hold for every utterance at any size
+    assert np.all(olens[:, 0] >= 0)
+    assert np.all(np.diff(scores, axis=1) <= 0)
+    assert st["frames"] == int(lens.sum()) and st["joins"] >= st["frames"]
+    om = oracle_model(m)
+    for b in sample:
+        got = nbest_from_arrays(tokens, olens, scores, b)
+        ok, why, _ = check_against_oracle(om, enc[b, :lens[b]], cfg.N, S, 4 * S + 16, got)
+        assert ok, "%s utterance %d: %s" % (name, b, why)
+
+
+def test_full_batch_bf16_c3_top1_sampled():
+    cfg = tw_synth.get_config("c3")
+    S, T = 3, 240
+    m, enc, lens, (tokens, olens, scores, status), st = _decode(cfg, S, 1, T)
+    assert st["limit_hits"] == 0
+    om = oracle_model(m)
+    agree = 0
+    sample = (1, 64, 127)
+    for b in sample:
+        got = nbest_from_arrays(tokens, olens, scores, b)
+        ref, _ = tws.token_wise_beam_search(om, enc[b, :lens[b]], cfg.N, S, max_iters=4 * S + 16)
+        agree += got[0][0] == ref[0][0]
+        assert abs(got[0][1] - ref[0][1]) < 1.0
+    print("c3 bf16 top-1 agreement on sampled utterances: %d/%d" % (agree, len(sample)))
+    assert agree >= 2
