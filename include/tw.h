@@ -233,6 +233,13 @@ int tw_joiner_expand_noalloc(const float* W_out, const float* b_out, int32_t J, 
                              int32_t G, int32_t R, float* out_ldphi, float* out_ldnb, float* out_la,
                              void* stream);
 
+/* TW_MODE_BF16 only: switches between the fused joiner (joiner, softmax, Eq. 3-7 and the first stage
+ * of ChooseNBestExpansions in one kernel, logits kept in tensor memory; the default whenever
+ * S <= 32 and V is a multiple of 256 up to 4096) and the staged kernels that pass the logits through
+ * device memory.  Both compute the same quantities.  TW_ERR_STATE if the fused kernel is not
+ * available for this handle. */
+int tw_set_fused(tw_handle* h, int on);
+
 /* Per-stage device timing of tw_decode with CUDA events on the decode stream (adds two event records
  * per stage per step); off by default. */
 int tw_set_profiling(tw_handle* h, int on);

@@ -11,7 +11,7 @@ TW_OK, TW_ERR_ARG, TW_ERR_ALLOC, TW_ERR_CUDA, TW_ERR_LIMIT, TW_ERR_STATE, TW_ERR
 
 EXPORTED_SYMBOLS = [
     "tw_init", "tw_destroy", "tw_decode", "tw_decode_host", "tw_max_tokens", "tw_project_encoder",
-    "tw_joiner_segment", "tw_expand", "tw_joiner_expand", "tw_predictor_step", "tw_get_stats", "tw_set_profiling",
+    "tw_joiner_segment", "tw_expand", "tw_joiner_expand", "tw_predictor_step", "tw_get_stats", "tw_set_profiling", "tw_set_fused",
     "tw_joiner_expand_noalloc",
     "tw_last_cuda_error", "tw_strerror",
 ]
@@ -68,6 +68,7 @@ def load_library() -> C.CDLL:
     lib.tw_predictor_step.argtypes = [vp, vp, vp, i32, vp, vp, vp]
     lib.tw_get_stats.argtypes = [vp, C.POINTER(_Stats)]
     lib.tw_set_profiling.argtypes = [vp, C.c_int]
+    lib.tw_set_fused.argtypes = [vp, C.c_int]
     lib.tw_joiner_expand_noalloc.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp]
     lib.tw_last_cuda_error.argtypes = [vp]
     lib.tw_strerror.argtypes = [C.c_int]
@@ -240,6 +241,10 @@ class TwDecoder:
         self._check(self.lib.tw_predictor_step(self.h, tokens.data_ptr(), _ptr(state_in), R, _ptr(state_out), Pp.data_ptr(),
                                                self._stream()), "tw_predictor_step")
         return state_out, Pp
+
+    def set_fused(self, on: bool) -> bool:
+        """tw_set_fused; returns False when the fused kernel is not available for this handle."""
+        return self.lib.tw_set_fused(self.h, int(bool(on))) == TW_OK
 
     def set_profiling(self, on: bool):
         self._check(self.lib.tw_set_profiling(self.h, int(bool(on))), "tw_set_profiling")

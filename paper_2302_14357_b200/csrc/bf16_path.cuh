@@ -45,4 +45,27 @@ void launch_gather_concat_bf16(const float* src1, const int* idx1, long long ld1
 // joiner A operand: A[(r, t), j] = tanh(E[e0[r]+t, j] + Pp[p[r], j]) as bf16; zero rows for padding frames
 void launch_joiner_A_bf16(const JoinerRows& rows, __nv_bfloat16* A, cudaStream_t st);
 
+
+// ---- fused joiner + softmax + Eq. 3-7 + candidate selection (fused_joiner.cu) ------------------
+struct FusedJoinerParams {
+  const int* R_dev; int R_max;       // hypothesis rows (device count optional)
+  int S, V, K, blank, CL, N;         // CL = V / 256 CTAs per cluster; K = J
+  const float* bias;                 // b_out [V]
+  const float* ld_old;               // [R][S]
+  const int* row_slen;               // [R] (nullptr: S)
+  float* ldphi; float* la; float* lse;   // [R], [R][S], [R][S]
+  float* ldnb;                       // optional [R][V]: every delta_nb (stage output; decode leaves it null)
+  float* c2v; int* c2k; int* c2n;    // per-CTA candidate lists [R][32][kMaxBeam], [R][32]
+  int* err;
+};
+bool fused_joiner_eligible(int S, int V, int J);
+long long fused_joiner_A_rows(int R_max, int S);      // rows of the tile-layout A operand
+int fused_joiner_setup(int CL, int* max_clusters);
+void launch_joiner_A_tiled(const JoinerRows& rows, __nv_bfloat16* A, cudaStream_t st);
+int launch_fused_joiner(const CUtensorMap& tmA, const CUtensorMap& tmB256, const FusedJoinerParams& p,
+                        int max_clusters, float* cand_v, int* cand_k, int* cand_n, cudaStream_t st);
+// adds log J(t, parent row, token) to A_ld of the hypotheses created in this step
+void launch_survivor_ld(const HypState& hs, int B, const __nv_bfloat16* A, const __nv_bfloat16* W, const float* bias,
+                        const float* lse, cudaStream_t st);
+
 }  // namespace tw

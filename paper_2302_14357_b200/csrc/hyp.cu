@@ -264,17 +264,21 @@ __global__ void __launch_bounds__(kStepThreads) hyp_step_kernel(HypState hs) {
       hs.new_slot[b * kMaxBeam + i] = (int)gn;
       hs.new_par[b * kMaxBeam + i] = (int)gp;
       hs.new_tok[b * kMaxBeam + i] = k;
+      hs.new_row[b * kMaxBeam + i] = r0 + h;
       hs.A_slot[b * kMaxBeam + i] = s_keep_slot[i];
       hs.A_ls[b * kMaxBeam + i] = s_keep_ls[i];
     }
     const long long r = r0 + h;
     for (int t = lane; t < S; t += 32) {
       double v = -INFINITY;
-      if (t < slen && hs.logp != nullptr) {
+      if (t < slen) {
         const double a = hs.la_d ? hs.la_d[r * S + t] : (double)hs.la[r * S + t];
-        double lj = (double)hs.logp[(r * S + t) * V + k];
-        if (hs.lse) lj -= (double)hs.lse[r * S + t];
-        v = s_Als[h] + a + lj;
+        v = s_Als[h] + a;
+        if (hs.logp != nullptr) {      // otherwise log J(t, k) is added by a follow-up kernel
+          double lj = (double)hs.logp[(r * S + t) * V + k];
+          if (hs.lse) lj -= (double)hs.lse[r * S + t];
+          v += lj;
+        }
       }
       hs.A_ld[((long long)b * kMaxBeam + i) * S + t] = v;
     }

@@ -173,6 +173,21 @@ int build_bf16(tw_handle* h) {
       TW_TRY(make_bf16_mat(h, &h->bf.X[l], nullptr, h->R_max, 2 * h->Hd, true, false));
     }
   }
+  // fused joiner: needs S frames of a hypothesis inside one warp and V split into 256-column CTAs
+  if (fused_joiner_eligible(h->S, h->V, h->J)) {
+    h->bf.CL = h->V / 256;
+    int s = fused_joiner_setup(h->bf.CL, &h->bf.max_clusters);
+    if (s == TW_OK) {
+      TW_TRY(make_bf16_mat(h, &h->bf.A_tiled, nullptr, fused_joiner_A_rows(h->R_max, h->S), h->J, true, false));
+      TW_TRY(dev_alloc(h, &h->bf.lse, (size_t)h->R_max * h->S));
+      TW_TRY(dev_alloc(h, &h->bf.c2v, (size_t)h->R_max * 32 * kMaxBeam));
+      TW_TRY(dev_alloc(h, &h->bf.c2k, (size_t)h->R_max * 32 * kMaxBeam));
+      TW_TRY(dev_alloc(h, &h->bf.c2n, (size_t)h->R_max * 32));
+      h->bf.fused_ok = h->bf.fused_on = true;
+    }
+  }
+  h->hs_fused = h->hs;
+  h->hs_fused.logp = nullptr; h->hs_fused.lse = nullptr; h->hs_fused.ldphi_d = nullptr; h->hs_fused.la_d = nullptr;
   TW_CUDA(h, cudaGetLastError());
   return TW_OK;
 }
@@ -210,6 +225,7 @@ int build_workspace(tw_handle* h) {
   TW_TRY(dev_alloc(h, &hs.new_slot, nb * kMaxBeam));
   TW_TRY(dev_alloc(h, &hs.new_par, nb * kMaxBeam));
   TW_TRY(dev_alloc(h, &hs.new_tok, nb * kMaxBeam));
+  TW_TRY(dev_alloc(h, &hs.new_row, nb * kMaxBeam));
   int** per_row[] = {&hs.row_b, &hs.row_e0, &hs.row_p, &hs.row_slen, &hs.pw_new, &hs.pw_par, &hs.pw_tok,
                      &h->stage_e0, &h->stage_slen};
   for (int** p : per_row) TW_TRY(dev_alloc(h, p, R));
@@ -317,6 +333,19 @@ void enqueue_scan(tw_handle* h, const JoinerRows& rows, const float* ld_old, flo
   }
 }
 
+// Fused path: joiner, softmax, Eq. 3-7 and per-row candidates with the logits kept in tensor memory
+int enqueue_joiner_fused(tw_handle* h, const JoinerRows& rows, const float* ld_old, float* ldphi, float* ldnb,
+                         float* la, const CandOut& cand, cudaStream_t st, int* launches) {
+  launch_joiner_A_tiled(rows, h->bf.A_tiled.ptr, st);
+  FusedJoinerParams fp{};
+  fp.R_dev = rows.R_dev; fp.R_max = rows.R_max; fp.S = rows.S; fp.V = rows.V; fp.K = rows.J; fp.blank = h->blank;
+  fp.CL = h->bf.CL; fp.N = h->N; fp.bias = h->b_out; fp.ld_old = ld_old; fp.row_slen = rows.row_slen;
+  fp.ldphi = ldphi; fp.la = la; fp.lse = h->bf.lse; fp.ldnb = ldnb;
+  fp.c2v = h->bf.c2v; fp.c2k = h->bf.c2k; fp.c2n = h->bf.c2n; fp.err = h->bf.err;
+  *launches += cand.n ? 3 : 2;
+  return launch_fused_joiner(h->bf.A_tiled.as_A, h->bf.W_out.as_B256, fp, h->bf.max_clusters, cand.v, cand.k, cand.n, st);
+}
+
 // z[(r, t), :] = W_out tanh(E + Pp) + b_out into `logp` (rows of padding frames hold no result)
 void enqueue_joiner_logits(tw_handle* h, const JoinerRows& rows, float* logp, cudaStream_t st, int* launches) {
   if (h->mode == TW_MODE_BF16) {
@@ -376,6 +405,13 @@ int tw_destroy(tw_handle* h) {
 
 int tw_max_tokens(const tw_handle* h) { return h ? h->U_cap : -1; }
 int tw_last_cuda_error(const tw_handle* h) { return h ? h->last_cuda : 0; }
+
+int tw_set_fused(tw_handle* h, int on) {
+  if (!h) return TW_ERR_ARG;
+  if (on && !h->bf.fused_ok) return TW_ERR_STATE;
+  h->bf.fused_on = on != 0;
+  return TW_OK;
+}
 
 int tw_set_profiling(tw_handle* h, int on) {
   if (!h) return TW_ERR_ARG;

@@ -20,6 +20,7 @@ struct tw_handle {
   float* init_Pp = nullptr;   // and its projected output [J]
 
   tw::HypState hs{};
+  tw::HypState hs_fused{};    // same arrays, but log J is not materialised (fused joiner path)
   float* E = nullptr;         // projected encoder frames [max_batch * max_T, J]
   float* gates = nullptr;     // LSTM gate pre-activations [R_max, 4 Hd]
   int *stage_e0 = nullptr, *stage_slen = nullptr;   // [R_max] scratch of the stage entry points
@@ -33,6 +34,12 @@ struct tw_handle {
     tw::Bf16Mat Htop;                                     // [R_max, Hd]
     float* EmbProj = nullptr;   // [V, 4Hd] = emb W_ih[0]^T + b[0]: layer 0's input half, one row per token
     int* err = nullptr;                                   // device error word of the bounded waits
+    // fused joiner + softmax + Eq. 3-7 + selection (logits stay in tensor memory)
+    bool fused_ok = false, fused_on = false;
+    int CL = 0, max_clusters = 0;
+    tw::Bf16Mat A_tiled;                                  // A operand in the fused kernel's tile layout
+    float* lse = nullptr;                                 // [R_max, S]
+    float* c2v = nullptr; int* c2k = nullptr; int* c2n = nullptr;   // per-CTA candidate lists
   } bf;
 
   // staging of tw_decode_host (allocated on first use)
@@ -54,6 +61,8 @@ struct tw_handle {
 namespace tw {
 // stages shared by tw_decode and the stage entry points
 void enqueue_joiner_logits(tw_handle* h, const JoinerRows& rows, float* logp, cudaStream_t st, int* launches);
+int enqueue_joiner_fused(tw_handle* h, const JoinerRows& rows, const float* ld_old, float* ldphi, float* ldnb,
+                         float* la, const CandOut& cand, cudaStream_t st, int* launches);
 void enqueue_scan(tw_handle* h, const JoinerRows& rows, const float* ld_old, float* logp, float* ldphi,
                   float* ldnb, float* la, double* ldphi_d, double* la_d, const CandOut& cand, cudaStream_t st,
                   int* launches);

@@ -116,7 +116,7 @@ struct HypState {
   float* slot_hc;   // [B*capSlot][L][2][Hd]   (LSTM predictor only)
   float* slot_Pp;   // [B*capSlot][J]          (LSTM predictor only)
   // new hypotheses of the current step, per utterance: [B][kMaxBeam] (global slot ids)
-  int *new_slot, *new_par, *new_tok;
+  int *new_slot, *new_par, *new_tok, *new_row;   // new_row: joiner row of the parent
   // compacted rows of the current step: [B*N]
   int *row_b, *row_e0, *row_p, *row_slen; float* row_ld;   // row_ld [R][S]
   int *row_off, *new_off;     // [B] first row / first work-list entry of each utterance

@@ -78,6 +78,65 @@ def test_predictor_step_bf16(layers, hidden):
         np.testing.assert_allclose(Pp[r], om.W_p @ o, atol=BF16_STAGE_TOL)
 
 
+@pytest.mark.parametrize("V,J,S,R", [(256, 64, 3, 5), (256, 128, 1, 40), (1024, 640, 3, 45), (4096, 1024, 2, 70),
+                                     (512, 64, 10, 13), (768, 128, 5, 30), (2048, 256, 32, 9)])
+def test_joiner_expand_fused_bf16(V, J, S, R):
+    """The fused kernel (logits in tensor memory, statistics exchanged across the cluster) against the
+    oracle's joiner -> softmax -> Eq. 3-7 chain, ragged segments, and against the staged kernels."""
+    from oracle import segment_math as sm
+    cfg = _cfg(V=V, J=J)
+    m, dec = _decoder(cfg, S, N=4, max_batch=(R + 3) // 4, max_T=64)
+    assert dec.set_fused(True)
+    om = oracle_model(m)
+    rng = np.random.default_rng(V + R + S)
+    G = 4
+    enc = tw_synth.round_to_bf16(rng.standard_normal((G, S, cfg.D_enc)).astype(np.float32))
+    row_group = rng.integers(0, G, size=R).astype(np.int32)
+    seg_len = np.array([S, max(1, S - 1), S, max(1, S // 2)], np.int32)
+    pred = rng.standard_normal((R, cfg.P)).astype(np.float32) * 0.5
+    ld_old = (rng.standard_normal((R, S)) - 2).astype(np.float32)
+    ld_old[0, 1:] = -np.inf
+    E = dec.project_encoder(enc).reshape(G, S, J)
+    Pp = (pred.astype(np.float64) @ om.W_p.T).astype(np.float32)
+    fused = [x.cpu().numpy() for x in dec.joiner_expand(E, Pp, row_group, seg_len, ld_old)]
+    assert dec.set_fused(False)
+    staged = [x.cpu().numpy() for x in dec.joiner_expand(E, Pp, row_group, seg_len, ld_old)]
+    for r in range(R):
+        sl = seg_len[row_group[r]]
+        lj = rm.joiner_log_probs(om, enc[row_group[r], :sl], pred[r:r + 1])
+        lo = ld_old[r:r + 1, :sl].astype(np.float64)
+        lBl = sm.blank_product(lj)
+        ld = sm.nonblank_expansion_t(lj, lBl, lo)
+        ref_nb = sm.nonblank_expansion(ld)[0]
+        ref_phi = sm.blank_expansion(lBl, lo)[0]
+        for got in (fused, staged):
+            assert abs(got[0][r] - ref_phi) < BF16_STAGE_TOL
+            fin = np.isfinite(got[1][r])
+            assert np.isneginf(got[1][r][0]) and fin[1:].all()
+            assert np.abs(got[1][r][fin] - ref_nb[fin]).max() < BF16_STAGE_TOL
+            la = got[2][r]
+            assert np.all(np.isneginf(la[sl:]))
+    np.testing.assert_allclose(fused[0], staged[0], atol=5e-3)
+
+
+def test_decode_fused_equals_staged_bf16():
+    """Same N-best from the fused joiner and from the staged kernels on a small model."""
+    from paper_2302_14357_b200.binding import MODE_BF16, TwDecoder, weights_from_synth
+    cfg = _cfg(batch=6, T=40, V=512)
+    m = tw_synth.make_model(cfg)
+    enc, lens = tw_synth.make_encoder_batch(cfg)
+    dec = TwDecoder(weights_from_synth(m), N=cfg.N, S=3, mode=MODE_BF16, max_batch=6, max_T=40)
+    assert dec.set_fused(True)
+    a = [x.cpu().numpy() for x in dec.decode(enc, lens)[:4]]
+    sa = dec.stats()
+    assert dec.set_fused(False)
+    b = [x.cpu().numpy() for x in dec.decode(enc, lens)[:4]]
+    same_top1 = sum(int(np.array_equal(a[0][u, 0], b[0][u, 0])) for u in range(6))
+    assert same_top1 >= 5
+    np.testing.assert_allclose(a[2][:, 0], b[2][:, 0], atol=0.05)
+    assert sa["calls"] > 0 and np.all(a[3] == 0)
+
+
 def _top1_agreement(cfg, S, batch, T):
     from paper_2302_14357_b200.binding import MODE_BF16, TwDecoder, weights_from_synth
     m = tw_synth.make_model(cfg)
