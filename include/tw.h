@@ -104,6 +104,7 @@ typedef struct {
   int64_t ns_scan;       /* softmax and Eq. 3-7 where they are separate kernels        */
   int64_t ns_hyp;        /* AddAndMerge, threshold, N-best expansions, compaction      */
   int64_t joiner_launches; /* launches summed in ns_joiner                             */
+  int64_t fused_clusters;  /* clusters the fused joiner keeps resident (0: fused path unavailable) */
 } tw_stats;
 
 /* Builds a decoder: copies (and in bf16 mode converts) the weights, runs InitPredictor, allocates
@@ -234,8 +235,8 @@ int tw_joiner_expand_noalloc(const float* W_out, const float* b_out, int32_t J, 
                              void* stream);
 
 /* TW_MODE_BF16 only: switches between the fused joiner (joiner, softmax, Eq. 3-7 and the first stage
- * of ChooseNBestExpansions in one kernel, logits kept in tensor memory; the default whenever
- * S <= 32 and V is a multiple of 256 up to 4096) and the staged kernels that pass the logits through
+ * of ChooseNBestExpansions in one kernel, logits kept in tensor memory; available when S <= 32 and V is a
+ * multiple of 256 up to 4096, and the default for S <= 5) and the staged kernels that pass the logits through
  * device memory.  Both compute the same quantities.  TW_ERR_STATE if the fused kernel is not
  * available for this handle. */
 int tw_set_fused(tw_handle* h, int on);

@@ -49,21 +49,25 @@ void launch_joiner_A_bf16(const JoinerRows& rows, __nv_bfloat16* A, cudaStream_t
 // ---- fused joiner + softmax + Eq. 3-7 + candidate selection (fused_joiner.cu) ------------------
 struct FusedJoinerParams {
   const int* R_dev; int R_max;       // hypothesis rows (device count optional)
-  int S, V, K, blank, CL, N;         // CL = V / 256 CTAs per cluster; K = J
+  int S, V, K, blank, CL;            // CL = V / 256 CTAs per cluster; K = J
+  int no_max;                        // logits are bounded (|z| <= 40): softmax sums need no maximum
   const float* bias;                 // b_out [V]
   const float* ld_old;               // [R][S]
   const int* row_slen;               // [R] (nullptr: S)
   float* ldphi; float* la; float* lse;   // [R], [R][S], [R][S]
-  float* ldnb;                       // optional [R][V]: every delta_nb (stage output; decode leaves it null)
-  float* c2v; int* c2k; int* c2n;    // per-CTA candidate lists [R][32][kMaxBeam], [R][32]
+  float* ldnb;                       // [R][V] delta_nb as a probability ratio, NOT its log (0 at the blank column)
   int* err;
 };
 bool fused_joiner_eligible(int S, int V, int J);
 long long fused_joiner_A_rows(int R_max, int S);      // rows of the tile-layout A operand
-int fused_joiner_setup(int CL, int* max_clusters);
+int fused_joiner_setup(int CL, int S, int* max_clusters);
+// max_k (sum_j |W_out[k, j]| + |b_out[k]|): bound of |z| since |tanh| <= 1; written to *out (device)
+void launch_logit_bound(const __nv_bfloat16* W, const float* bias, int V, int J, float* out, cudaStream_t st);
+// in place: x -> log x (log 0 = -inf), n elements
+void launch_log_inplace(float* x, long long n, cudaStream_t st);
 void launch_joiner_A_tiled(const JoinerRows& rows, __nv_bfloat16* A, cudaStream_t st);
 int launch_fused_joiner(const CUtensorMap& tmA, const CUtensorMap& tmB256, const FusedJoinerParams& p,
-                        int max_clusters, float* cand_v, int* cand_k, int* cand_n, cudaStream_t st);
+                        int max_clusters, cudaStream_t st);
 // adds log J(t, parent row, token) to A_ld of the hypotheses created in this step
 void launch_survivor_ld(const HypState& hs, int B, const __nv_bfloat16* A, const __nv_bfloat16* W, const float* bias,
                         const float* lse, cudaStream_t st);

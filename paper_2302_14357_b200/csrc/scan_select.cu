@@ -51,11 +51,23 @@ __global__ void __launch_bounds__(kMaxT) scan_select_kernel(ScanSelectArgs a) {
   const int r = blockIdx.x;
   if (r >= R) return;
   const int S = a.S, V = a.V, blank = a.blank;
-  const int sl = a.row_slen ? a.row_slen[r] : S;
+  const int sl = a.dnb_in ? 1 : (a.row_slen ? a.row_slen[r] : S);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int kT = blockDim.x, nwarps = kT >> 5, ngroups = kT >> 4;
   const float* z = a.z + (long long)r * S * V;
 
+  float tmax = -INFINITY;
+  if (a.dnb_in != nullptr) {
+    // selection only: the row of delta_nb values is given
+    const float* src = a.dnb_in + (long long)r * V;
+    for (int k = tid; k < V; k += kT) {
+      float v = src[k];
+      if (a.dnb_linear) v = v > 0.f ? v : -INFINITY;     // order is the same as that of the logs
+      zs[k] = v; tmax = fmaxf(tmax, v);
+    }
+    if (tid == 0) s_nsurv = 0;
+    __syncthreads();
+  } else {
   // ---- the one pass over global memory
   if ((V & 3) == 0) {
     const int n4 = sl * V / 4;
@@ -108,7 +120,6 @@ __global__ void __launch_bounds__(kMaxT) scan_select_kernel(ScanSelectArgs a) {
   __syncthreads();
 
   // ---- delta_nb for every token; kept in shared memory (frame 0's logits are no longer needed)
-  float tmax = -INFINITY;
   for (int k = tid; k < V; k += kT) {
     float out = -INFINITY;
     if (k != blank) {
@@ -123,6 +134,7 @@ __global__ void __launch_bounds__(kMaxT) scan_select_kernel(ScanSelectArgs a) {
     if (sl > 0) zs[k] = out;                 // only this thread ever touches column k
     if (a.ldnb) a.ldnb[(long long)r * V + k] = out;
     tmax = fmaxf(tmax, out);
+  }
   }
   if (a.cand.n == nullptr) return;
   const int N = a.cand.N;
@@ -164,7 +176,10 @@ __global__ void __launch_bounds__(kMaxT) scan_select_kernel(ScanSelectArgs a) {
         const float v = s_sv[i]; const int k = s_sk[i];
         int rank = 0;
         for (int j = 0; j < ns; ++j) rank += cand_better(s_sv[j], s_sk[j], v, k);
-        if (rank < N) { a.cand.v[(long long)r * kMaxBeam + rank] = v; a.cand.k[(long long)r * kMaxBeam + rank] = k; }
+        if (rank < N) {
+          a.cand.v[(long long)r * kMaxBeam + rank] = a.dnb_linear ? __logf(v) : v;
+          a.cand.k[(long long)r * kMaxBeam + rank] = k;
+        }
       }
       if (lane == 0) a.cand.n[r] = min(ns, N);
     }
@@ -197,7 +212,7 @@ __global__ void __launch_bounds__(kMaxT) scan_select_kernel(ScanSelectArgs a) {
       }
       bv = __shfl_sync(0xffffffffu, bv, 0); bk = __shfl_sync(0xffffffffu, bk, 0); bl = __shfl_sync(0xffffffffu, bl, 0);
       if (bv == -INFINITY) break;
-      if (lane == 0) { a.cand.v[(long long)r * kMaxBeam + j] = bv; a.cand.k[(long long)r * kMaxBeam + j] = bk; }
+      if (lane == 0) { a.cand.v[(long long)r * kMaxBeam + j] = a.dnb_linear ? __logf(bv) : bv; a.cand.k[(long long)r * kMaxBeam + j] = bk; }
       if (lane == bl) ++pos;
       ++cnt;
     }
@@ -219,7 +234,7 @@ int scan_select_setup() {
 
 void launch_scan_select(const ScanSelectArgs& a, bool fast_math, cudaStream_t st) {
   if (a.R_max <= 0) return;
-  const size_t smem = scan_select_smem_bytes(a.S, a.V);
+  const size_t smem = a.dnb_in ? scan_select_smem_bytes(1, a.V) : scan_select_smem_bytes(a.S, a.V);
   // a row that takes most of an SM's shared memory runs alone there: give it the whole SM's threads
   const int threads = smem > 96 * 1024 ? 1024 : (smem > 48 * 1024 ? 512 : 256);
   if (fast_math) scan_select_kernel<true><<<a.R_max, threads, smem, st>>>(a);

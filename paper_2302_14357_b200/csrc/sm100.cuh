@@ -80,6 +80,17 @@ __device__ __forceinline__ void st_cluster_f32x2(uint32_t addr, float a, float b
 __device__ __forceinline__ void st_cluster_f32(uint32_t addr, float a) {
   asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(a) : "memory");
 }
+// Asynchronous stores into another CTA's shared memory that signal `bytes written` on an mbarrier of
+// that CTA (both addresses from map_to_cta with the same rank): the receiver arms the barrier with
+// mbar_expect_tx and waits on it; no fence or separate arrival is needed.
+__device__ __forceinline__ void st_async_f32x2(uint32_t addr, float a, float b, uint32_t remote_bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];"
+               ::"r"(addr), "f"(a), "f"(b), "r"(remote_bar) : "memory");
+}
+__device__ __forceinline__ void st_async_f32(uint32_t addr, float a, uint32_t remote_bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.f32 [%0], %1, [%2];"
+               ::"r"(addr), "f"(a), "r"(remote_bar) : "memory");
+}
 __device__ __forceinline__ void fence_acq_rel_cluster() { asm volatile("fence.acq_rel.cluster;" ::: "memory"); }
 // arrive on an mbarrier of another CTA of the cluster (address from map_to_cta), releasing prior writes
 __device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {

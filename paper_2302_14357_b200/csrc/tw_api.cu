@@ -176,14 +176,20 @@ int build_bf16(tw_handle* h) {
   // fused joiner: needs S frames of a hypothesis inside one warp and V split into 256-column CTAs
   if (fused_joiner_eligible(h->S, h->V, h->J)) {
     h->bf.CL = h->V / 256;
-    int s = fused_joiner_setup(h->bf.CL, &h->bf.max_clusters);
+    int s = fused_joiner_setup(h->bf.CL, h->S, &h->bf.max_clusters);
     if (s == TW_OK) {
+      // |z| <= max_k (|W_out[k, :]|_1 + |b_out[k]|) because |tanh| <= 1: small enough => sum exp(z) needs no max
+      float* bound_dev = nullptr; float bound = 0.f;
+      TW_TRY(dev_alloc(h, &bound_dev, (size_t)1));
+      launch_logit_bound(h->bf.W_out.ptr, h->b_out, h->V, h->J, bound_dev, 0);
+      TW_CUDA(h, cudaMemcpy(&bound, bound_dev, sizeof(float), cudaMemcpyDeviceToHost));
+      h->bf.no_max = (bound <= 40.f);
       TW_TRY(make_bf16_mat(h, &h->bf.A_tiled, nullptr, fused_joiner_A_rows(h->R_max, h->S), h->J, true, false));
       TW_TRY(dev_alloc(h, &h->bf.lse, (size_t)h->R_max * h->S));
-      TW_TRY(dev_alloc(h, &h->bf.c2v, (size_t)h->R_max * 32 * kMaxBeam));
-      TW_TRY(dev_alloc(h, &h->bf.c2k, (size_t)h->R_max * 32 * kMaxBeam));
-      TW_TRY(dev_alloc(h, &h->bf.c2n, (size_t)h->R_max * 32));
-      h->bf.fused_ok = h->bf.fused_on = true;
+      TW_TRY(scan_select_setup());
+      h->bf.fused_ok = true;
+      // default: on for the short segments the kernel is specialised for; longer ones are currently faster staged
+      h->bf.fused_on = h->S <= 5;
     }
   }
   h->hs_fused = h->hs;
@@ -337,13 +343,21 @@ void enqueue_scan(tw_handle* h, const JoinerRows& rows, const float* ld_old, flo
 int enqueue_joiner_fused(tw_handle* h, const JoinerRows& rows, const float* ld_old, float* ldphi, float* ldnb,
                          float* la, const CandOut& cand, cudaStream_t st, int* launches) {
   launch_joiner_A_tiled(rows, h->bf.A_tiled.ptr, st);
+  if (ldnb == nullptr) ldnb = h->hs.ldnb;
   FusedJoinerParams fp{};
   fp.R_dev = rows.R_dev; fp.R_max = rows.R_max; fp.S = rows.S; fp.V = rows.V; fp.K = rows.J; fp.blank = h->blank;
-  fp.CL = h->bf.CL; fp.N = h->N; fp.bias = h->b_out; fp.ld_old = ld_old; fp.row_slen = rows.row_slen;
-  fp.ldphi = ldphi; fp.la = la; fp.lse = h->bf.lse; fp.ldnb = ldnb;
-  fp.c2v = h->bf.c2v; fp.c2k = h->bf.c2k; fp.c2n = h->bf.c2n; fp.err = h->bf.err;
-  *launches += cand.n ? 3 : 2;
-  return launch_fused_joiner(h->bf.A_tiled.as_A, h->bf.W_out.as_B256, fp, h->bf.max_clusters, cand.v, cand.k, cand.n, st);
+  fp.CL = h->bf.CL; fp.no_max = h->bf.no_max ? 1 : 0; fp.bias = h->b_out; fp.ld_old = ld_old; fp.row_slen = rows.row_slen;
+  fp.ldphi = ldphi; fp.la = la; fp.lse = h->bf.lse; fp.ldnb = ldnb; fp.err = h->bf.err;
+  TW_TRY(launch_fused_joiner(h->bf.A_tiled.as_A, h->bf.W_out.as_B256, fp, h->bf.max_clusters, st));
+  *launches += 2;
+  if (cand.n != nullptr) {      // ChooseNBestExpansions, first stage: the rows' N best tokens
+    ScanSelectArgs a{};
+    a.R_dev = rows.R_dev; a.R_max = rows.R_max; a.S = rows.S; a.V = rows.V; a.blank = h->blank;
+    a.cand = cand; a.dnb_in = ldnb; a.dnb_linear = 1;
+    launch_scan_select(a, true, st);
+    *launches += 1;
+  }
+  return TW_OK;
 }
 
 // z[(r, t), :] = W_out tanh(E + Pp) + b_out into `logp` (rows of padding frames hold no result)
@@ -422,6 +436,7 @@ int tw_set_profiling(tw_handle* h, int on) {
 int tw_get_stats(const tw_handle* h, tw_stats* out) {
   if (!h || !out) return TW_ERR_ARG;
   *out = h->stats;
+  out->fused_clusters = h->bf.fused_ok ? h->bf.max_clusters : 0;
   return TW_OK;
 }
 

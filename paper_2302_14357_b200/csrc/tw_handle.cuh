@@ -35,11 +35,10 @@ struct tw_handle {
     float* EmbProj = nullptr;   // [V, 4Hd] = emb W_ih[0]^T + b[0]: layer 0's input half, one row per token
     int* err = nullptr;                                   // device error word of the bounded waits
     // fused joiner + softmax + Eq. 3-7 + selection (logits stay in tensor memory)
-    bool fused_ok = false, fused_on = false;
+    bool fused_ok = false, fused_on = false, no_max = false;
     int CL = 0, max_clusters = 0;
     tw::Bf16Mat A_tiled;                                  // A operand in the fused kernel's tile layout
     float* lse = nullptr;                                 // [R_max, S]
-    float* c2v = nullptr; int* c2k = nullptr; int* c2n = nullptr;   // per-CTA candidate lists
   } bf;
 
   // staging of tw_decode_host (allocated on first use)

@@ -85,6 +85,8 @@ struct ScanSelectArgs {
   float* lse_out;      // [R, S] softmax normalisers: log J(t, k) = z[t, k] - lse[t]
   float *ldphi, *ldnb, *la; double *ldphi_d, *la_d;
   CandOut cand;
+  const float* dnb_in = nullptr;   // when set: [R, V] delta_nb values are given and only the selection runs
+  int dnb_linear = 0;              // dnb_in holds probabilities (0 = none), candidates are returned as logs
 };
 bool scan_select_fits(int S, int V);   // the row's S x V logits fit in shared memory
 int scan_select_setup();
