@@ -30,6 +30,25 @@ __global__ void gather_concat_bf16_kernel(const float* __restrict__ src1, const 
   for (int k = threadIdx.x; k < K; k += blockDim.x) d[k] = __float2bfloat16_rn(k < K1 ? a[k] : b[k - K1]);
 }
 
+__global__ void gather_parents_bf16_kernel(GatherParents g, const int* n_dev, int n_max) {
+  const int n = n_dev ? *n_dev : n_max;
+  const int r = blockIdx.x, l = blockIdx.y;
+  if (r >= n) return;
+  const float* src = g.hc + (long long)(g.idx ? g.idx[r] : r) * g.stride + (long long)l * 2 * g.Hd;
+  __nv_bfloat16* d = g.dst[l] + (long long)r * g.ld[l] + g.off[l];
+  for (int k = threadIdx.x * 2; k < g.Hd; k += blockDim.x * 2)
+    *reinterpret_cast<__nv_bfloat162*>(d + k) = __floats2bfloat162_rn(src[k], src[k + 1]);
+}
+
+__global__ void permute_cols_f32_kernel(const float* __restrict__ src, const int* __restrict__ perm, long long rows,
+                                        int cols, float* __restrict__ dst) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= rows * cols) return;
+  const long long r = i / cols;
+  const int c = (int)(i - r * cols);
+  dst[i] = src[r * cols + perm[c]];
+}
+
 __device__ __forceinline__ float tanh_fast(float x) {
   float y;
   asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -67,6 +86,16 @@ void launch_gather_concat_bf16(const float* src1, const int* idx1, long long ld1
                                __nv_bfloat16* dst, cudaStream_t st) {
   if (n_max <= 0) return;
   gather_concat_bf16_kernel<<<n_max, 256, 0, st>>>(src1, idx1, ld1, K1, src2, idx2, ld2, K2, n_dev, n_max, dst);
+}
+
+void launch_gather_parents_bf16(const GatherParents& g, const int* n_dev, int n_max, cudaStream_t st) {
+  if (n_max <= 0 || g.L <= 0) return;
+  gather_parents_bf16_kernel<<<dim3(n_max, g.L), 128, 0, st>>>(g, n_dev, n_max);
+}
+
+void launch_permute_cols_f32(const float* src, const int* perm, long long rows, int cols, float* dst, cudaStream_t st) {
+  const long long n = rows * cols;
+  if (n > 0) permute_cols_f32_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(src, perm, rows, cols, dst);
 }
 
 void launch_joiner_A_bf16(const JoinerRows& rows, __nv_bfloat16* A, cudaStream_t st) {

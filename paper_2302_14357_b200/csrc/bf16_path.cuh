@@ -7,6 +7,18 @@
 
 namespace tw {
 
+// LSTM cell epilogue of a gate GEMM whose output columns are interleaved by unit (column 4 j + g is
+// gate g of hidden unit j, gates in the order input, forget, cell, output):
+//   c' = sigma(f) c + sigma(i) tanh(g),  h' = sigma(o) tanh(c')
+// c is read from state row (idx_in ? idx_in[m] : m) of hc_in, (h', c') are written to state row
+// (idx_out ? idx_out[m] : m) of hc_out (rows are [L][2][Hd]), and h' also goes, as bf16, to row m of
+// xnext (the next GEMM's A operand).
+struct LstmEpi {
+  const float* hc_in; const int* idx_in; float* hc_out; const int* idx_out;
+  int L, l, Hd;
+  __nv_bfloat16* xnext; long long ld_xnext;
+};
+
 struct GemmBf16Params {
   const int* M_dev;   // device row count (nullptr: use M); CTAs beyond it exit
   int M, N, K;        // M is the maximum when M_dev is given
@@ -18,6 +30,8 @@ struct GemmBf16Params {
   const float* addend = nullptr;   // optional: row m also gets addend[(add_idx ? add_idx[m] : m) * ld_add + n]
   const int* add_idx = nullptr;
   long long ld_add = 0;
+  int epi = 0;        // 0: store C (+ bias, + addend); 1: LSTM cell (C is not written)
+  LstmEpi lstm = {};
 };
 
 // 2-D bf16 tensor map over a row-major [rows, K] matrix, box = 64 x box_rows, 128-byte swizzle.
@@ -42,6 +56,15 @@ void launch_f32_to_bf16(const float* src, __nv_bfloat16* dst, long long n, cudaS
 void launch_gather_concat_bf16(const float* src1, const int* idx1, long long ld1, int K1, const float* src2,
                                const int* idx2, long long ld2, int K2, const int* n_dev, int n_max,
                                __nv_bfloat16* dst, cudaStream_t st);
+// X[l][r, off_l : off_l + Hd] = bf16(h of layer l in state row (idx ? idx[r] : r)), for every layer at once
+struct GatherParents {
+  const float* hc; const int* idx; long long stride;   // state rows [L][2][Hd]
+  int L, Hd;
+  __nv_bfloat16* dst[kMaxLayers]; int ld[kMaxLayers]; int off[kMaxLayers];
+};
+void launch_gather_parents_bf16(const GatherParents& g, const int* n_dev, int n_max, cudaStream_t st);
+// dst[r, c] = src[r, perm[c]]  (fp32, rows x cols)
+void launch_permute_cols_f32(const float* src, const int* perm, long long rows, int cols, float* dst, cudaStream_t st);
 // joiner A operand: A[(r, t), j] = tanh(E[e0[r]+t, j] + Pp[p[r], j]) as bf16; zero rows for padding frames
 void launch_joiner_A_bf16(const JoinerRows& rows, __nv_bfloat16* A, cudaStream_t st);
 

@@ -25,7 +25,14 @@ struct Cfg {
   static constexpr size_t kSmem = (size_t)kStages * (kABytes + kBBytes) + 1024 + 256;
 };
 
-template <int BN>
+__device__ __forceinline__ float sigmoid_fast(float x) { return __fdividef(1.f, 1.f + __expf(-x)); }
+__device__ __forceinline__ float tanh_fast_g(float x) {
+  float y;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+template <int BN, int EPI>
 __global__ void __launch_bounds__(kThreadsGemm, 1)
 gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmBf16Params p) {
   using C = Cfg<BN>;
@@ -121,9 +128,18 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       const int m = m0 + q * 32 + lane;
       float* crow = nullptr;
       const float* arow = nullptr;           // optional per-row addend (gathered)
+      const float* cin = nullptr;            // LSTM epilogue: parent's c, new (h, c), bf16 copy of h
+      float* hout = nullptr;
+      __nv_bfloat16* xrow = nullptr;
       if (m < M) {
-        crow = p.C + (long long)(p.oidx ? p.oidx[m] : m) * p.ldC;
+        if (EPI == 0) crow = p.C + (long long)(p.oidx ? p.oidx[m] : m) * p.ldC;
         if (p.addend) arow = p.addend + (long long)(p.add_idx ? p.add_idx[m] : m) * p.ld_add;
+        if (EPI == 1) {
+          const long long stride = (long long)p.lstm.L * 2 * p.lstm.Hd, lo = (long long)p.lstm.l * 2 * p.lstm.Hd;
+          cin = p.lstm.hc_in + (long long)(p.lstm.idx_in ? p.lstm.idx_in[m] : m) * stride + lo + p.lstm.Hd;
+          hout = p.lstm.hc_out + (long long)(p.lstm.idx_out ? p.lstm.idx_out[m] : m) * stride + lo;
+          xrow = p.lstm.xnext + (long long)m * p.lstm.ld_xnext;
+        }
       }
 #pragma unroll 1
       for (int c = 0; c < kColsPerWarp / 32; ++c) {
@@ -131,7 +147,37 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const int col = half * kColsPerWarp + c * 32;
         tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + buf * BN + (uint32_t)col, v);
         const int nb = n0 + col;
-        if (crow != nullptr && nb < p.N) {
+        if (EPI == 1) {
+          if (hout != nullptr && nb < p.N) {       // N = 4 Hd is a multiple of 32: the chunk is 8 whole units
+            if (p.bias) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) v[j] += p.bias[nb + j];
+            }
+            if (arow) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) v[j] += arow[nb + j];
+            }
+            const int j0 = nb >> 2;
+            float hn[8], cn[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+              const float c = sigmoid_fast(v[4 * u + 1]) * cin[j0 + u] + sigmoid_fast(v[4 * u]) * tanh_fast_g(v[4 * u + 2]);
+              cn[u] = c;
+              hn[u] = sigmoid_fast(v[4 * u + 3]) * tanh_fast_g(c);
+            }
+            float* cout = hout + p.lstm.Hd;
+            *reinterpret_cast<float4*>(hout + j0) = make_float4(hn[0], hn[1], hn[2], hn[3]);
+            *reinterpret_cast<float4*>(hout + j0 + 4) = make_float4(hn[4], hn[5], hn[6], hn[7]);
+            *reinterpret_cast<float4*>(cout + j0) = make_float4(cn[0], cn[1], cn[2], cn[3]);
+            *reinterpret_cast<float4*>(cout + j0 + 4) = make_float4(cn[4], cn[5], cn[6], cn[7]);
+            __nv_bfloat162 b0 = __floats2bfloat162_rn(hn[0], hn[1]), b1 = __floats2bfloat162_rn(hn[2], hn[3]);
+            __nv_bfloat162 b2 = __floats2bfloat162_rn(hn[4], hn[5]), b3 = __floats2bfloat162_rn(hn[6], hn[7]);
+            uint4 pk;
+            pk.x = *reinterpret_cast<uint32_t*>(&b0); pk.y = *reinterpret_cast<uint32_t*>(&b1);
+            pk.z = *reinterpret_cast<uint32_t*>(&b2); pk.w = *reinterpret_cast<uint32_t*>(&b3);
+            *reinterpret_cast<uint4*>(xrow + j0) = pk;
+          }
+        } else if (crow != nullptr && nb < p.N) {
           if (nb + 32 <= p.N && ((reinterpret_cast<uintptr_t>(crow + nb) & 15) == 0)) {
             if (p.bias) {
 #pragma unroll
@@ -193,9 +239,11 @@ int make_tmap_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint64_t K
 }
 
 int gemm_bf16_setup() {
-  cudaError_t e1 = cudaFuncSetAttribute(gemm_bf16_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<256>::kSmem);
-  cudaError_t e2 = cudaFuncSetAttribute(gemm_bf16_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<128>::kSmem);
-  return (e1 == cudaSuccess && e2 == cudaSuccess) ? TW_OK : TW_ERR_CUDA;
+  cudaError_t e1 = cudaFuncSetAttribute(gemm_bf16_kernel<256, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<256>::kSmem);
+  cudaError_t e2 = cudaFuncSetAttribute(gemm_bf16_kernel<128, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<128>::kSmem);
+  cudaError_t e3 = cudaFuncSetAttribute(gemm_bf16_kernel<256, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<256>::kSmem);
+  cudaError_t e4 = cudaFuncSetAttribute(gemm_bf16_kernel<128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<128>::kSmem);
+  return (e1 == cudaSuccess && e2 == cudaSuccess && e3 == cudaSuccess && e4 == cudaSuccess) ? TW_OK : TW_ERR_CUDA;
 }
 
 void launch_gemm_bf16(const CUtensorMap& tmA, const CUtensorMap& tmB128, const CUtensorMap& tmB256,
@@ -212,11 +260,13 @@ void launch_gemm_bf16(const CUtensorMap& tmA, const CUtensorMap& tmB128, const C
   // small problems: narrower tiles put more SMs to work
   if ((long long)mt * nt256 >= num_sms) {
     const int grid = (int)((long long)mt * nt256 < num_sms ? mt * nt256 : num_sms);
-    gemm_bf16_kernel<256><<<grid, kThreadsGemm, Cfg<256>::kSmem, st>>>(tmA, tmB256, p);
+    if (p.epi == 1) gemm_bf16_kernel<256, 1><<<grid, kThreadsGemm, Cfg<256>::kSmem, st>>>(tmA, tmB256, p);
+    else gemm_bf16_kernel<256, 0><<<grid, kThreadsGemm, Cfg<256>::kSmem, st>>>(tmA, tmB256, p);
   } else {
     const long long tiles = (long long)mt * nt128;
     const int grid = (int)(tiles < num_sms ? tiles : num_sms);
-    gemm_bf16_kernel<128><<<grid, kThreadsGemm, Cfg<128>::kSmem, st>>>(tmA, tmB128, p);
+    if (p.epi == 1) gemm_bf16_kernel<128, 1><<<grid, kThreadsGemm, Cfg<128>::kSmem, st>>>(tmA, tmB128, p);
+    else gemm_bf16_kernel<128, 0><<<grid, kThreadsGemm, Cfg<128>::kSmem, st>>>(tmA, tmB128, p);
   }
 }
 

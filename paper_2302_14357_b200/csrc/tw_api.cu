@@ -1,5 +1,6 @@
 // C ABI of libtw: handle life-cycle, the decode driver and the separately callable stages.
 #include <new>
+#include <vector>
 #include <stdio.h>
 #include <string.h>
 
@@ -75,43 +76,45 @@ void enqueue_predictor(tw_handle* h, const int* tok, const float* hc_in, const i
   }
   const int L = h->L, Hd = h->Hd;
   const long long stride = (long long)L * 2 * Hd;
+  if (h->mode == TW_MODE_BF16) {
+    // parents' h of every layer -> the recurrent halves of the layers' A operands (one launch)
+    GatherParents g{};
+    g.hc = hc_in; g.idx = idx_in; g.stride = stride; g.L = L; g.Hd = Hd;
+    for (int l = 0; l < L; ++l) { g.dst[l] = h->bf.X[l].ptr; g.ld[l] = (int)h->bf.X[l].K; g.off[l] = (l == 0) ? 0 : Hd; }
+    launch_gather_parents_bf16(g, n_dev, n_max, st);
+    // gate GEMMs with the LSTM cell in the epilogue; each writes the next GEMM's input half as bf16
+    for (int l = 0; l < L; ++l) {
+      GemmBf16Params p{n_dev, n_max, 4 * Hd, (int)h->bf.X[l].K, nullptr, nullptr, 0, nullptr, h->bf.err};
+      if (l == 0) { p.addend = h->bf.EmbProj; p.add_idx = tok; p.ld_add = 4 * Hd; }   // W_ih[0] emb[tok] + b[0]: a table row
+      else p.bias = h->bf.bias_perm[l];
+      p.epi = 1;
+      p.lstm = LstmEpi{hc_in, idx_in, hc_out, idx_out, L, l, Hd,
+                       (l + 1 < L) ? h->bf.X[l + 1].ptr : h->bf.Htop.ptr, (l + 1 < L) ? 2LL * Hd : (long long)Hd};
+      launch_gemm_bf16(h->bf.X[l].as_A, h->bf.W_cat[l].as_B128, h->bf.W_cat[l].as_B256, p, st);
+    }
+    gemm_bf16(h, h->bf.Htop, h->bf.W_p, n_dev, n_max, Pp_out, idx_out, h->J, nullptr, st);
+    *launches += L + 2;
+    return;
+  }
   for (int l = 0; l < L; ++l) {
     const float* x = (l == 0) ? h->emb : hc_out + (long long)(l - 1) * 2 * Hd;
     const int* xi = (l == 0) ? tok : idx_out;
     const long long xld = (l == 0) ? h->emb_dim : stride;
     const int xk = (l == 0) ? h->emb_dim : Hd;
     const float* hp = hc_in + (long long)l * 2 * Hd;
-    if (h->mode == TW_MODE_BF16 && l == 0) {
-      // the input half W_ih[0] emb[tok] + b[0] is a table row; only W_hh[0] h_parent is contracted
-      launch_gather_concat_bf16(hp, idx_in, stride, Hd, nullptr, nullptr, 0, 0, n_dev, n_max, h->bf.X[0].ptr, st);
-      gemm_bf16(h, h->bf.X[0], h->bf.W_cat[0], n_dev, n_max, h->gates, nullptr, 4 * Hd, nullptr, st, h->bf.EmbProj,
-                tok, 4 * Hd);
-      *launches += 1;
-    } else if (h->mode == TW_MODE_BF16) {
-      launch_gather_concat_bf16(x, xi, xld, xk, hp, idx_in, stride, Hd, n_dev, n_max, h->bf.X[l].ptr, st);
-      gemm_bf16(h, h->bf.X[l], h->bf.W_cat[l], n_dev, n_max, h->gates, nullptr, 4 * Hd, h->b_l[l], st);
-      *launches += 1;
-    } else {
-      GemmOperand xo{x, xi, xld, h->W_ih[l], xk, xk};
-      GemmOperand ro{hp, idx_in, stride, h->W_hh[l], Hd, Hd};
-      GemmOut o{h->gates, nullptr, 4 * Hd, h->b_l[l]};
-      launch_gemm_f32(xo, ro, o, n_dev, n_max, 4 * Hd, st);
-    }
+    GemmOperand xo{x, xi, xld, h->W_ih[l], xk, xk};
+    GemmOperand ro{hp, idx_in, stride, h->W_hh[l], Hd, Hd};
+    GemmOut o{h->gates, nullptr, 4 * Hd, h->b_l[l]};
+    launch_gemm_f32(xo, ro, o, n_dev, n_max, 4 * Hd, st);
     // pointwise: c' = sigma(f) c + sigma(i) tanh(g), h' = sigma(o) tanh(c')
     launch_lstm_pointwise(h->gates, idx_out, idx_in, n_dev, n_max, hc_in, hc_out, L, l, Hd, st);
     *launches += 2;
   }
   const float* top = hc_out + (long long)(L - 1) * 2 * Hd;
-  if (h->mode == TW_MODE_BF16) {
-    launch_gather_concat_bf16(top, idx_out, stride, Hd, nullptr, nullptr, 0, 0, n_dev, n_max, h->bf.Htop.ptr, st);
-    gemm_bf16(h, h->bf.Htop, h->bf.W_p, n_dev, n_max, Pp_out, idx_out, h->J, nullptr, st);
-    *launches += 2;
-  } else {
-    GemmOperand to{top, idx_out, stride, h->W_p, h->P, h->P};
-    GemmOut o{Pp_out, idx_out, h->J, nullptr};
-    launch_gemm_f32(to, none, o, n_dev, n_max, h->J, st);
-    *launches += 1;
-  }
+  GemmOperand to{top, idx_out, stride, h->W_p, h->P, h->P};
+  GemmOut o{Pp_out, idx_out, h->J, nullptr};
+  launch_gemm_f32(to, none, o, n_dev, n_max, h->J, st);
+  *launches += 1;
 }
 
 int enqueue_predictor_plain(tw_handle* h, const int* tokens, const float* state_in, int R,
@@ -156,21 +159,38 @@ int build_bf16(tw_handle* h) {
   if (h->pred_kind == TW_PRED_LSTM) {
     TW_TRY(make_bf16_mat(h, &h->bf.W_p, h->W_p, h->J, h->P, false, true));
     TW_TRY(make_bf16_mat(h, &h->bf.Htop, nullptr, h->R_max, h->Hd, true, false));
+    // Gate GEMM outputs are interleaved by hidden unit (column 4 j + g = gate g of unit j) so that the
+    // LSTM cell can run in the GEMM epilogue: weight rows, biases and the table are permuted once here.
+    const int G4 = 4 * h->Hd;
+    std::vector<int> perm(G4);
+    for (int j = 0; j < h->Hd; ++j)
+      for (int g = 0; g < 4; ++g) perm[4 * j + g] = g * h->Hd + j;
+    int* perm_dev = nullptr;
+    TW_TRY(dev_alloc(h, &perm_dev, (size_t)G4));
+    TW_CUDA(h, cudaMemcpy(perm_dev, perm.data(), G4 * sizeof(int), cudaMemcpyHostToDevice));
     {
-      // EmbProj[k] = W_ih[0] emb[k] + b[0]  (fp32 products of the stored weights, exact inputs)
-      TW_TRY(dev_alloc(h, &h->bf.EmbProj, (size_t)h->V * 4 * h->Hd));
+      // EmbProj[k] = W_ih[0] emb[k] + b[0]  (fp32 products of the stored weights, exact inputs), columns permuted
+      float* tmp = nullptr;
+      TW_CUDA(h, cudaMalloc((void**)&tmp, (size_t)h->V * G4 * sizeof(float)));
+      TW_TRY(dev_alloc(h, &h->bf.EmbProj, (size_t)h->V * G4));
       GemmOperand a{h->emb, nullptr, h->emb_dim, h->W_ih[0], h->emb_dim, h->emb_dim};
       GemmOperand none{};
-      GemmOut o{h->bf.EmbProj, nullptr, 4 * h->Hd, h->b_l[0]};
-      launch_gemm_f32(a, none, o, nullptr, h->V, 4 * h->Hd, 0);
-      TW_TRY(make_bf16_mat(h, &h->bf.W_cat[0], h->W_hh[0], 4 * h->Hd, h->Hd, false, true));
+      GemmOut o{tmp, nullptr, G4, h->b_l[0]};
+      launch_gemm_f32(a, none, o, nullptr, h->V, G4, 0);
+      launch_permute_cols_f32(tmp, perm_dev, h->V, G4, h->bf.EmbProj, 0);
+      TW_CUDA(h, cudaDeviceSynchronize());
+      cudaFree(tmp);
+      TW_TRY(make_bf16_mat(h, &h->bf.W_cat[0], nullptr, G4, h->Hd, false, true));
+      launch_gather_concat_bf16(h->W_hh[0], perm_dev, h->Hd, h->Hd, nullptr, nullptr, 0, 0, nullptr, G4, h->bf.W_cat[0].ptr, 0);
       TW_TRY(make_bf16_mat(h, &h->bf.X[0], nullptr, h->R_max, h->Hd, true, false));
     }
     for (int l = 1; l < h->L; ++l) {
-      TW_TRY(make_bf16_mat(h, &h->bf.W_cat[l], nullptr, 4 * h->Hd, 2 * h->Hd, false, true));
-      launch_gather_concat_bf16(h->W_ih[l], nullptr, h->Hd, h->Hd, h->W_hh[l], nullptr, h->Hd, h->Hd, nullptr, 4 * h->Hd,
+      TW_TRY(make_bf16_mat(h, &h->bf.W_cat[l], nullptr, G4, 2 * h->Hd, false, true));
+      launch_gather_concat_bf16(h->W_ih[l], perm_dev, h->Hd, h->Hd, h->W_hh[l], perm_dev, h->Hd, h->Hd, nullptr, G4,
                                 h->bf.W_cat[l].ptr, 0);
       TW_TRY(make_bf16_mat(h, &h->bf.X[l], nullptr, h->R_max, 2 * h->Hd, true, false));
+      TW_TRY(dev_alloc(h, &h->bf.bias_perm[l], (size_t)G4));
+      launch_permute_cols_f32(h->b_l[l], perm_dev, 1, G4, h->bf.bias_perm[l], 0);
     }
   }
   // fused joiner: needs S frames of a hypothesis inside one warp and V split into 256-column CTAs

@@ -32,6 +32,7 @@ struct tw_handle {
     tw::Bf16Mat A_join;                                   // [R_max * S, J]  tanh(E + Pp)
     tw::Bf16Mat X[tw::kMaxLayers];                        // LSTM layer inputs: [R_max, Hd] (layer 0: parent h) or [R_max, 2Hd]
     tw::Bf16Mat Htop;                                     // [R_max, Hd]
+    float* bias_perm[tw::kMaxLayers] = {};   // LSTM biases in the interleaved gate order (layers > 0)
     float* EmbProj = nullptr;   // [V, 4Hd] = emb W_ih[0]^T + b[0]: layer 0's input half, one row per token
     int* err = nullptr;                                   // device error word of the bounded waits
     // fused joiner + softmax + Eq. 3-7 + selection (logits stay in tensor memory)
