@@ -60,10 +60,22 @@ __global__ void __launch_bounds__(kMaxT) scan_select_kernel(ScanSelectArgs a) {
   if (a.dnb_in != nullptr) {
     // selection only: the row of delta_nb values is given
     const float* src = a.dnb_in + (long long)r * V;
-    for (int k = tid; k < V; k += kT) {
-      float v = src[k];
-      if (a.dnb_linear) v = v > 0.f ? v : -INFINITY;     // order is the same as that of the logs
-      zs[k] = v; tmax = fmaxf(tmax, v);
+    if ((V & 3) == 0) {
+      for (int k = tid * 4; k < V; k += kT * 4) {
+        float4 v = *reinterpret_cast<const float4*>(src + k);
+        if (a.dnb_linear) {                                // order is the same as that of the logs
+          v.x = v.x > 0.f ? v.x : -INFINITY; v.y = v.y > 0.f ? v.y : -INFINITY;
+          v.z = v.z > 0.f ? v.z : -INFINITY; v.w = v.w > 0.f ? v.w : -INFINITY;
+        }
+        *reinterpret_cast<float4*>(zs + k) = v;
+        tmax = fmaxf(fmaxf(tmax, fmaxf(v.x, v.y)), fmaxf(v.z, v.w));
+      }
+    } else {
+      for (int k = tid; k < V; k += kT) {
+        float v = src[k];
+        if (a.dnb_linear) v = v > 0.f ? v : -INFINITY;
+        zs[k] = v; tmax = fmaxf(tmax, v);
+      }
     }
     if (tid == 0) s_nsurv = 0;
     __syncthreads();
