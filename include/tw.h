@@ -236,7 +236,7 @@ int tw_joiner_expand_noalloc(const float* W_out, const float* b_out, int32_t J, 
 
 /* TW_MODE_BF16 only: switches between the fused joiner (joiner, softmax, Eq. 3-7 and the first stage
  * of ChooseNBestExpansions in one kernel, logits kept in tensor memory; available when S <= 32 and V is a
- * multiple of 256 up to 4096, and the default for S <= 5) and the staged kernels that pass the logits through
+ * multiple of 256 up to 4096, and the default for S in {1..5, 8, 10}) and the staged kernels that pass the logits through
  * device memory.  Both compute the same quantities.  TW_ERR_STATE if the fused kernel is not
  * available for this handle. */
 int tw_set_fused(tw_handle* h, int on);

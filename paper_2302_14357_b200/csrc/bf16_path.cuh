@@ -82,6 +82,7 @@ struct FusedJoinerParams {
   int* err;
 };
 bool fused_joiner_eligible(int S, int V, int J);
+bool fused_joiner_specialised(int S);   // a kernel instance with this segment size compiled in exists
 long long fused_joiner_A_rows(int R_max, int S);      // rows of the tile-layout A operand
 int fused_joiner_setup(int CL, int S, int* max_clusters);
 // max_k (sum_j |W_out[k, j]| + |b_out[k]|): bound of |z| since |tanh| <= 1; written to *out (device)

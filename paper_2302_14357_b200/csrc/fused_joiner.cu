@@ -64,17 +64,21 @@ __device__ __forceinline__ float logaddexp_fast(float a, float b) {
 // ST > 0: segment size known at compile time (plain unrolled shuffles); ST == 0: any S <= 32.
 template <int ST>
 __device__ __forceinline__ float window_sum(float x, int S) {
-  if (ST > 0) {
+  if (ST > 0 && ST <= 4) {
     float total = x;
 #pragma unroll
     for (int d = 1; d < ST; ++d) total += __shfl_down_sync(0xffffffffu, x, d);
     return total;
   }
+  // doubling: windows of 1, 2, 4, ... lanes; the set bits of S pick the pieces (unrolled when S is known)
+  const int SS = ST > 0 ? ST : S;
   float total = 0.f, cur = x;
   int off = 0;
-  for (int size = 1; size <= S; size <<= 1) {
-    if (S & size) { total += __shfl_down_sync(0xffffffffu, cur, off); off += size; }
-    cur += __shfl_down_sync(0xffffffffu, cur, size);
+#pragma unroll
+  for (int size = 1; size <= 32; size <<= 1) {
+    if (size > SS) break;
+    if (SS & size) { total += __shfl_down_sync(0xffffffffu, cur, off); off += size; }
+    if (2 * size <= SS) cur += __shfl_down_sync(0xffffffffu, cur, size);
   }
   return total;
 }

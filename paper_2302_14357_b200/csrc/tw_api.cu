@@ -208,8 +208,9 @@ int build_bf16(tw_handle* h) {
       TW_TRY(dev_alloc(h, &h->bf.lse, (size_t)h->R_max * h->S));
       TW_TRY(scan_select_setup());
       h->bf.fused_ok = true;
-      // default: on for the short segments the kernel is specialised for; longer ones are currently faster staged
-      h->bf.fused_on = h->S <= 5;
+      // default: on for the segment sizes with a specialised kernel instance; the generic instance is
+      // currently slower than the staged kernels
+      h->bf.fused_on = fused_joiner_specialised(h->S);
     }
   }
   h->hs_fused = h->hs;
