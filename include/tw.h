@@ -100,11 +100,12 @@ typedef struct {
   /* device time per stage in nanoseconds, summed over the decode; zero unless tw_set_profiling(h, 1) */
   int64_t ns_prologue;   /* E = enc W_e^T and list initialisation                      */
   int64_t ns_predictor;  /* UpdatePredictorOutput                                      */
-  int64_t ns_joiner;     /* joiner contraction (+ softmax and Eq. 3-7 where fused)     */
-  int64_t ns_scan;       /* softmax and Eq. 3-7 where they are separate kernels        */
+  int64_t ns_joiner;     /* the joiner kernel alone: contraction, or the fused contraction + softmax + Eq. 3-7 */
+  int64_t ns_scan;       /* separate softmax / Eq. 3-7 / selection kernels and the joiner's operand kernel */
   int64_t ns_hyp;        /* AddAndMerge, threshold, N-best expansions, compaction      */
   int64_t joiner_launches; /* launches summed in ns_joiner                             */
   int64_t fused_clusters;  /* clusters the fused joiner keeps resident (0: fused path unavailable) */
+  int64_t fused_on;        /* 1 if tw_decode takes the fused joiner path                          */
 } tw_stats;
 
 /* Builds a decoder: copies (and in bf16 mode converts) the weights, runs InitPredictor, allocates

@@ -38,7 +38,7 @@ class _Config(C.Structure):
 
 class _Stats(C.Structure):
     _fields_ = [(n, C.c_int64) for n in ("frames", "calls", "joins", "steps", "rows", "kernel_launches", "limit_hits", "joiner_frame_rows",
-                                          "ns_prologue", "ns_predictor", "ns_joiner", "ns_scan", "ns_hyp", "joiner_launches", "fused_clusters")]
+                                          "ns_prologue", "ns_predictor", "ns_joiner", "ns_scan", "ns_hyp", "joiner_launches", "fused_clusters", "fused_on")]
 
 
 def lib_path() -> str:

@@ -362,14 +362,16 @@ void enqueue_scan(tw_handle* h, const JoinerRows& rows, const float* ld_old, flo
 
 // Fused path: joiner, softmax, Eq. 3-7 and per-row candidates with the logits kept in tensor memory
 int enqueue_joiner_fused(tw_handle* h, const JoinerRows& rows, const float* ld_old, float* ldphi, float* ldnb,
-                         float* la, const CandOut& cand, cudaStream_t st, int* launches) {
+                         float* la, const CandOut& cand, cudaStream_t st, int* launches, StageMarkFn mark_fn) {
   launch_joiner_A_tiled(rows, h->bf.A_tiled.ptr, st);
+  if (mark_fn) mark_fn(h, 3, st);       // operand preparation is booked with the elementwise stages
   if (ldnb == nullptr) ldnb = h->hs.ldnb;
   FusedJoinerParams fp{};
   fp.R_dev = rows.R_dev; fp.R_max = rows.R_max; fp.S = rows.S; fp.V = rows.V; fp.K = rows.J; fp.blank = h->blank;
   fp.CL = h->bf.CL; fp.no_max = h->bf.no_max ? 1 : 0; fp.bias = h->b_out; fp.ld_old = ld_old; fp.row_slen = rows.row_slen;
   fp.ldphi = ldphi; fp.la = la; fp.lse = h->bf.lse; fp.ldnb = ldnb; fp.err = h->bf.err;
   TW_TRY(launch_fused_joiner(h->bf.A_tiled.as_A, h->bf.W_out.as_B256, fp, h->bf.max_clusters, st));
+  if (mark_fn) mark_fn(h, 2, st);       // the fused kernel alone
   *launches += 2;
   if (cand.n != nullptr) {      // ChooseNBestExpansions, first stage: the rows' N best tokens
     ScanSelectArgs a{};
@@ -458,6 +460,7 @@ int tw_get_stats(const tw_handle* h, tw_stats* out) {
   if (!h || !out) return TW_ERR_ARG;
   *out = h->stats;
   out->fused_clusters = h->bf.fused_ok ? h->bf.max_clusters : 0;
+  out->fused_on = (h->mode == TW_MODE_BF16 && h->bf.fused_on) ? 1 : 0;
   return TW_OK;
 }
 

@@ -61,8 +61,10 @@ struct tw_handle {
 namespace tw {
 // stages shared by tw_decode and the stage entry points
 void enqueue_joiner_logits(tw_handle* h, const JoinerRows& rows, float* logp, cudaStream_t st, int* launches);
+// mark_fn (optional) is called with stage 3 after the operand kernel and stage 2 after the fused kernel
+typedef void (*StageMarkFn)(tw_handle*, int, cudaStream_t);
 int enqueue_joiner_fused(tw_handle* h, const JoinerRows& rows, const float* ld_old, float* ldphi, float* ldnb,
-                         float* la, const CandOut& cand, cudaStream_t st, int* launches);
+                         float* la, const CandOut& cand, cudaStream_t st, int* launches, StageMarkFn mark_fn = nullptr);
 void enqueue_scan(tw_handle* h, const JoinerRows& rows, const float* ld_old, float* logp, float* ldphi,
                   float* ldnb, float* la, double* ldphi_d, double* la_d, const CandOut& cand, cudaStream_t st,
                   int* launches);
