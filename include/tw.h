@@ -242,6 +242,11 @@ int tw_joiner_expand_noalloc(const float* W_out, const float* b_out, int32_t J, 
  * available for this handle. */
 int tw_set_fused(tw_handle* h, int on);
 
+/* tw_decode replays its step body (16 device steps) as a CUDA graph, captured once per batch shape, on
+ * a stream of the handle's own that is ordered after `stream`; tw_set_graph(h, 0) makes it enqueue the
+ * kernels one by one on `stream` instead (as it also does while profiling is on).  Default: on. */
+int tw_set_graph(tw_handle* h, int on);
+
 /* Per-stage device timing of tw_decode with CUDA events on the decode stream (adds two event records
  * per stage per step); off by default. */
 int tw_set_profiling(tw_handle* h, int on);

@@ -435,6 +435,9 @@ int tw_destroy(tw_handle* h) {
   cudaDeviceSynchronize();
   for (void* p : h->dev_allocs) cudaFree(p);
   for (cudaEvent_t e : h->events) cudaEventDestroy(e);
+  if (h->graph_exec) cudaGraphExecDestroy(h->graph_exec);
+  if (h->ev_order) cudaEventDestroy(h->ev_order);
+  if (h->own_stream) cudaStreamDestroy(h->own_stream);
   if (h->host_flag) cudaFreeHost(h->host_flag);
   delete h;
   return TW_OK;
@@ -447,6 +450,12 @@ int tw_set_fused(tw_handle* h, int on) {
   if (!h) return TW_ERR_ARG;
   if (on && !h->bf.fused_ok) return TW_ERR_STATE;
   h->bf.fused_on = on != 0;
+  return TW_OK;
+}
+
+int tw_set_graph(tw_handle* h, int on) {
+  if (!h) return TW_ERR_ARG;
+  h->graph_on = on != 0;
   return TW_OK;
 }
 

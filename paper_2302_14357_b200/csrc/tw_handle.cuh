@@ -48,6 +48,15 @@ struct tw_handle {
 
   int* host_flag = nullptr;   // pinned copy of the device scalars
 
+  // The step body (kStepsPerGraph device steps) is captured once per (B, T, joiner path) into a CUDA
+  // graph and replayed; it runs on a stream of the handle's own because the caller's may be the legacy
+  // default stream, which cannot be captured.
+  bool graph_on = true, graph_failed = false;
+  cudaStream_t own_stream = nullptr;
+  cudaEvent_t ev_order = nullptr;
+  cudaGraphExec_t graph_exec = nullptr;
+  int graph_B = -1, graph_T = -1, graph_fused = -1, graph_launches = 0;
+
   // optional per-stage timing of tw_decode (tw_set_profiling): pooled events and the stage each closes
   bool profiling = false;
   std::vector<cudaEvent_t> events;
