@@ -119,6 +119,42 @@ def test_joiner_expand_fused_bf16(V, J, S, R):
     np.testing.assert_allclose(fused[0], staged[0], atol=5e-3)
 
 
+def test_fused_joiner_large_logits_online_maximum():
+    """Output weights large enough that the logits are not bounded by 40: the fused kernel must take its
+    running-maximum softmax path (the no-maximum shortcut is only valid for bounded logits)."""
+    from oracle import segment_math as sm
+    from paper_2302_14357_b200.binding import MODE_BF16, TwDecoder, weights_from_synth
+    cfg = _cfg(V=512, J=64)
+    m = tw_synth.make_model(cfg)
+    m.W_out = tw_synth.round_to_bf16(m.W_out * 16.0)          # sum_j |W_out[k, j]| is about 100
+    assert np.abs(m.W_out).sum(axis=1).max() > 60
+    S, R, G = 3, 11, 3
+    dec = TwDecoder(weights_from_synth(m), N=4, S=S, mode=MODE_BF16, max_batch=3, max_T=64)
+    assert dec.set_fused(True)
+    om = oracle_model(m)
+    rng = np.random.default_rng(2)
+    enc = tw_synth.round_to_bf16(rng.standard_normal((G, S, cfg.D_enc)).astype(np.float32))
+    row_group = rng.integers(0, G, size=R).astype(np.int32)
+    seg_len = np.array([3, 2, 3], np.int32)
+    pred = rng.standard_normal((R, cfg.P)).astype(np.float32) * 0.5
+    ld_old = (rng.standard_normal((R, S)) - 2).astype(np.float32)
+    E = dec.project_encoder(enc).reshape(G, S, cfg.J)
+    Pp = (pred.astype(np.float64) @ om.W_p.T).astype(np.float32)
+    ldphi, ldnb, la = [x.cpu().numpy() for x in dec.joiner_expand(E, Pp, row_group, seg_len, ld_old)]
+    for r in range(R):
+        sl = seg_len[row_group[r]]
+        lj = rm.joiner_log_probs(om, enc[row_group[r], :sl], pred[r:r + 1])
+        lo = ld_old[r:r + 1, :sl].astype(np.float64)
+        lBl = sm.blank_product(lj)
+        ref_nb = sm.nonblank_expansion(sm.nonblank_expansion_t(lj, lBl, lo))[0]
+        # logits of magnitude ~30 in bf16: the tolerance scales with them (2^-9 relative on the operands)
+        assert abs(ldphi[r] - sm.blank_expansion(lBl, lo)[0]) < 0.3
+        top = np.argsort(-ref_nb)[:8]
+        assert np.all(np.isfinite(ldnb[r][top]))
+        assert np.abs(ldnb[r][top] - ref_nb[top]).max() < 0.3
+        assert set(np.argsort(-ldnb[r])[:3]) & set(top[:5])
+
+
 def test_decode_fused_equals_staged_bf16():
     """Same N-best from the fused joiner and from the staged kernels on a small model."""
     from paper_2302_14357_b200.binding import MODE_BF16, TwDecoder, weights_from_synth
