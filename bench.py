@@ -82,7 +82,8 @@ def oracle_sample(cfg, S, frames, utt=0):
         cores = os.cpu_count() or 1
     m = tw_synth.make_model(cfg)
     enc, lens = tw_synth.make_encoder_batch(cfg, batch=utt + 1)
-    om = rm.RnntModel(m.W_e, m.W_p, m.W_out, m.b_out, m.emb, m.lstm_W_ih, m.lstm_W_hh, m.lstm_b)
+    om = rm.RnntModel(m.W_e, m.W_p, m.W_out, m.b_out, m.emb, m.lstm_W_ih, m.lstm_W_hh, m.lstm_b,
+                      activation=cfg.joiner_act)
     n = int(min(frames, lens[utt]))
     t0 = time.perf_counter()
     _, st = tws.token_wise_beam_search(om, enc[utt, :n], cfg.N, S, max_iters=4 * S + 16)
@@ -194,7 +195,7 @@ def run_ours(args, cfg, S):
     model = tw_synth.make_model(cfg)
     # every rank decodes its own batch of the same shape (utterances are independent: no exchange)
     enc_np, len_np = tw_synth.make_encoder_batch(cfg.with_(seed=cfg.seed + 1000 * rank), batch=B)
-    dec = TwDecoder(weights_from_synth(model), N=cfg.N, S=S, mode=mode, max_batch=B, max_T=cfg.T)
+    dec = TwDecoder(weights_from_synth(model), N=cfg.N, S=S, mode=mode, max_batch=B, max_T=cfg.T, joiner_act=cfg.joiner_act)
     if args.no_fused:
         dec.set_fused(False)
     enc = torch.from_numpy(enc_np).cuda()
@@ -206,15 +207,23 @@ def run_ours(args, cfg, S):
             dist.barrier()
         torch.cuda.synchronize()
 
+    # L2 hygiene: a workload whose inputs do not exceed L2 (126 MB) several times over gets L2 flushed
+    # (a 256 MB write) before every timed step, outside the timed interval
+    flush = None if enc_np.nbytes > 3 * 126e6 else torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+
     def timed(fn, steps):
         barrier()
-        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        ev0.record()
+        pairs = []
         for _ in range(steps):
-            fn()
-        ev1.record()
+            if flush is not None:
+                flush.zero_()
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ev0.record()
+            fn()                      # synchronous: tw_decode returns after its stream has drained
+            ev1.record()
+            pairs.append((ev0, ev1))
         barrier()
-        ms = ev0.elapsed_time(ev1)
+        ms = sum(a.elapsed_time(b) for a, b in pairs)
         if world > 1:
             t = torch.tensor([ms], device="cuda", dtype=torch.float64)
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -266,7 +275,8 @@ def run_ours(args, cfg, S):
         "ms_per_step": ms / args.steps, "ms_per_step_with_stage_events": ms_profiled / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": mode_name, "data": "synthetic",
         "config": {"workload": cfg.name, "B_per_gpu": B, "T": cfg.T, "N": cfg.N, "S": S, "J": cfg.J, "V": cfg.V,
-                   "mode": mode_name, "l2": "inputs larger than L2 (encoder batch %.0f MB, fresh per-step state)" % (enc_np.nbytes / 1e6),
+                   "mode": mode_name, "l2": ("inputs larger than L2 (encoder batch %.0f MB)" % (enc_np.nbytes / 1e6)) if flush is None
+                         else "L2 flushed by a 256 MB write before every timed step (encoder batch %.0f MB)" % (enc_np.nbytes / 1e6),
                    "parallelism": "independent utterance batches per GPU, no collective"},
         "calls_per_frame": st["calls"] / max(st["frames"], 1), "joins_per_frame": st["joins"] / max(st["frames"], 1),
         "device_steps_per_decode": st["steps"], "avg_rows_per_step": st["rows"] / max(st["steps"], 1),

@@ -44,13 +44,15 @@ typedef enum {
 
 enum { TW_MODE_F32 = 0, TW_MODE_BF16 = 1 };
 enum { TW_PRED_STATELESS = 0, TW_PRED_LSTM = 1 };
+enum { TW_ACT_TANH = 0, TW_ACT_RELU = 1 };   /* joiner hidden nonlinearity */
 
 #define TW_MAX_BEAM 16     /* N <= 16 */
 #define TW_MAX_SEGMENT 64  /* S <= 64 */
 
 /*
  * The RNN-T pieces the search calls (Sec. 3.1).
- *   joiner:    z(t,u,.) = W_out . tanh(W_e h_t + W_p g_u) + b_out,  J = softmax(z)
+ *   joiner:    z(t,u,.) = W_out . act(W_e h_t + W_p g_u) + b_out,  J = softmax(z); act = tanh, or ReLU
+ *              (the paper's models use "a ReLU layer followed by a single fully connected layer", Sec. 4.1)
  *   predictor: stateless  g = emb[last token]         (P == emb_dim; empty prefix -> emb[blank])
  *              LSTM       lstm_layers stacked cells, gate order (input, forget, cell, output),
  *                         one bias per layer, g = top layer's h   (P == lstm_hidden);
@@ -62,6 +64,7 @@ enum { TW_PRED_STATELESS = 0, TW_PRED_LSTM = 1 };
 typedef struct {
   int32_t D_enc, P, J, V, blank;
   int32_t pred_kind, emb_dim, lstm_layers, lstm_hidden;
+  int32_t joiner_act; /* TW_ACT_TANH or TW_ACT_RELU */
   const float* W_e;   /* [J, D_enc] */
   const float* W_p;   /* [J, P]     */
   const float* W_out; /* [V, J]     */

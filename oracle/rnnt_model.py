@@ -1,7 +1,8 @@
 """RNN-T model pieces the search calls (Sec. 3.1): joiner j(t,u,k) followed by
 softmax normalisation J, and the prediction network g(u).  fp64 throughout.
 
-Joiner form (synthetic workloads): z = W_out . tanh(W_e h_t + W_p g_u) + b_out.
+Joiner form: z = W_out . act(W_e h_t + W_p g_u) + b_out with act = tanh (the synthetic benchmark
+workloads) or ReLU (the paper's models: a ReLU layer followed by one fully connected layer, Sec. 4.1).
 Predictor: either stateless (g = embedding of the last token; the empty
 prefix uses the blank token's embedding) or a stack of LSTM layers with gate
 order (input, forget, cell, output) and a single bias per layer, started by
@@ -19,7 +20,7 @@ def _f64(x):
 class RnntModel:
     def __init__(self, W_e, W_p, W_out, b_out, emb,
                  lstm_W_ih: Sequence = (), lstm_W_hh: Sequence = (), lstm_b: Sequence = (),
-                 blank: int = 0):
+                 blank: int = 0, activation: str = "tanh"):
         self.W_e = _f64(W_e)        # [J, D_enc]
         self.W_p = _f64(W_p)        # [J, P]
         self.W_out = _f64(W_out)    # [V, J]
@@ -29,6 +30,8 @@ class RnntModel:
         self.lstm_W_hh = [_f64(w) for w in lstm_W_hh]   # [4Hd, Hd]
         self.lstm_b = [_f64(b) for b in lstm_b]         # [4Hd]
         self.blank = int(blank)
+        assert activation in ("tanh", "relu")
+        self.activation = activation
         self.V = self.W_out.shape[0]
         assert self.W_e.shape[0] == self.W_p.shape[0] == self.W_out.shape[1]
         assert len(self.lstm_W_ih) == len(self.lstm_W_hh) == len(self.lstm_b)
@@ -52,7 +55,8 @@ def joiner_log_probs(model: RnntModel, seg: np.ndarray, pred_out: np.ndarray) ->
     -> log J [H, S', V] for every (hypothesis, frame) pair."""
     e = _f64(seg) @ model.W_e.T                     # [S', J]
     p = _f64(pred_out) @ model.W_p.T                # [H, J]
-    hidden = np.tanh(e[None, :, :] + p[:, None, :])  # [H, S', J]
+    pre = e[None, :, :] + p[:, None, :]             # [H, S', J]
+    hidden = np.tanh(pre) if model.activation == "tanh" else np.maximum(pre, 0.0)
     z = hidden @ model.W_out.T + model.b_out        # [H, S', V]
     return log_softmax(z)
 

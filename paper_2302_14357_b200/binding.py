@@ -7,6 +7,7 @@ import numpy as np
 
 MODE_F32, MODE_BF16 = 0, 1
 PRED_STATELESS, PRED_LSTM = 0, 1
+ACT_TANH, ACT_RELU = 0, 1
 TW_OK, TW_ERR_ARG, TW_ERR_ALLOC, TW_ERR_CUDA, TW_ERR_LIMIT, TW_ERR_STATE, TW_ERR_TIMEOUT = range(7)
 
 EXPORTED_SYMBOLS = [
@@ -28,7 +29,7 @@ class TwError(RuntimeError):
 
 
 class _Model(C.Structure):
-    _fields_ = [(n, C.c_int32) for n in ("D_enc", "P", "J", "V", "blank", "pred_kind", "emb_dim", "lstm_layers", "lstm_hidden")] + \
+    _fields_ = [(n, C.c_int32) for n in ("D_enc", "P", "J", "V", "blank", "pred_kind", "emb_dim", "lstm_layers", "lstm_hidden", "joiner_act")] + \
                [(n, C.c_void_p) for n in ("W_e", "W_p", "W_out", "b_out", "emb", "host_lstm_W_ih", "host_lstm_W_hh", "host_lstm_b")]
 
 
@@ -97,7 +98,7 @@ class TwDecoder:
     float32 tensors ("lstm_W_ih", "lstm_W_hh", "lstm_b" are lists, one tensor per layer)."""
 
     def __init__(self, weights: Dict, N: int, S: int, mode: int = MODE_F32, max_batch: int = 1, max_T: int = 1,
-                 max_iters_per_segment: int = 0, max_tokens: int = 0, blank: int = 0):
+                 max_iters_per_segment: int = 0, max_tokens: int = 0, blank: int = 0, joiner_act: str = "tanh"):
         import torch
         self._torch = torch
         self.lib = load_library()
@@ -108,6 +109,8 @@ class TwDecoder:
         def dev(x):
             t = torch.as_tensor(x, dtype=torch.float32)
             return t.to(self.device).contiguous()
+        weights = dict(weights)
+        joiner_act = weights.pop("joiner_act", None) or joiner_act
         w = {k: ([dev(a) for a in v] if isinstance(v, (list, tuple)) else dev(v)) for k, v in weights.items() if v is not None}
         self._keep = w
         layers = len(w.get("lstm_W_ih", []))
@@ -120,6 +123,7 @@ class TwDecoder:
         m.pred_kind = PRED_LSTM if layers else PRED_STATELESS
         m.emb_dim, m.lstm_layers = emb_dim, layers
         m.lstm_hidden = w["lstm_W_hh"][0].shape[1] if layers else 0
+        m.joiner_act = {"tanh": ACT_TANH, "relu": ACT_RELU}[joiner_act]
         for name in ("W_e", "W_p", "W_out", "b_out", "emb"):
             setattr(m, name, w[name].data_ptr())
         self._tables = []
@@ -262,7 +266,8 @@ class TwDecoder:
 def weights_from_synth(m) -> Dict:
     """tw_model fields from a tw_synth.SyntheticModel (plain attribute access, no arithmetic)."""
     return dict(W_e=m.W_e, W_p=m.W_p, W_out=m.W_out, b_out=m.b_out, emb=m.emb,
-                lstm_W_ih=list(m.lstm_W_ih), lstm_W_hh=list(m.lstm_W_hh), lstm_b=list(m.lstm_b))
+                lstm_W_ih=list(m.lstm_W_ih), lstm_W_hh=list(m.lstm_W_hh), lstm_b=list(m.lstm_b),
+                joiner_act=m.cfg.joiner_act)
 
 
 NOALLOC_MAX_ROWS = 4096

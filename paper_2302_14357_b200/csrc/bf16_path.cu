@@ -70,7 +70,7 @@ __global__ void joiner_A_bf16_kernel(JoinerRows jr, __nv_bfloat16* __restrict__ 
   }
   const float* e = jr.E + (long long)(jr.row_e0[r] + t) * jr.J;
   const float* p = jr.Pp + (long long)(jr.row_p ? jr.row_p[r] : r) * jr.J;
-  for (int j = threadIdx.x; j < jr.J; j += blockDim.x) dst[j] = __float2bfloat16_rn(tanh_fast(e[j] + p[j]));
+  for (int j = threadIdx.x; j < jr.J; j += blockDim.x) dst[j] = __float2bfloat16_rn(jr.act == TW_ACT_RELU ? fmaxf(e[j] + p[j], 0.f) : tanh_fast(e[j] + p[j]));
 }
 
 }  // namespace

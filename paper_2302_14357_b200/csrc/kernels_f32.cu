@@ -98,7 +98,7 @@ __global__ void __launch_bounds__(256) gemm_f32_kernel(GemmParams p) {
         float q[4];
         load4(prow, k0 + kq, K, avalid, q);
 #pragma unroll
-        for (int i = 0; i < 4; ++i) a[i] = (avalid && k0 + kq + i < K) ? tanhf(a[i] + q[i]) : 0.f;
+        for (int i = 0; i < 4; ++i) a[i] = (avalid && k0 + kq + i < K) ? (p.jr.act == TW_ACT_RELU ? fmaxf(a[i] + q[i], 0.f) : tanhf(a[i] + q[i])) : 0.f;
       }
       load4(brow, k0 + kq, K, bvalid, b);
 #pragma unroll

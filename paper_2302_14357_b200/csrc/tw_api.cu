@@ -203,7 +203,7 @@ int build_bf16(tw_handle* h) {
       TW_TRY(dev_alloc(h, &bound_dev, (size_t)1));
       launch_logit_bound(h->bf.W_out.ptr, h->b_out, h->V, h->J, bound_dev, 0);
       TW_CUDA(h, cudaMemcpy(&bound, bound_dev, sizeof(float), cudaMemcpyDeviceToHost));
-      h->bf.no_max = (bound <= 40.f);
+      h->bf.no_max = (bound <= 40.f) && h->joiner_act == TW_ACT_TANH;   // the bound needs |act| <= 1
       TW_TRY(make_bf16_mat(h, &h->bf.A_tiled, nullptr, fused_joiner_A_rows(h->R_max, h->S), h->J, true, false));
       TW_TRY(dev_alloc(h, &h->bf.lse, (size_t)h->R_max * h->S));
       TW_TRY(scan_select_setup());
@@ -281,7 +281,7 @@ int build_workspace(tw_handle* h) {
 
 int init_impl(tw_handle* h, const tw_model* m, const tw_config* c) {
   h->D_enc = m->D_enc; h->P = m->P; h->J = m->J; h->V = m->V; h->blank = m->blank;
-  h->pred_kind = m->pred_kind; h->emb_dim = m->emb_dim;
+  h->pred_kind = m->pred_kind; h->emb_dim = m->emb_dim; h->joiner_act = m->joiner_act;
   h->L = (m->pred_kind == TW_PRED_LSTM) ? m->lstm_layers : 0;
   h->Hd = (m->pred_kind == TW_PRED_LSTM) ? m->lstm_hidden : 0;
   h->N = c->N; h->S = c->S; h->mode = c->mode; h->max_batch = c->max_batch; h->max_T = c->max_T;
@@ -405,6 +405,7 @@ int tw_init(const tw_model* m, const tw_config* c, tw_handle** out) {
   if (!m->W_e || !m->W_p || !m->W_out || !m->b_out || !m->emb) return TW_ERR_ARG;
   if (m->D_enc < 1 || m->P < 1 || m->J < 1 || m->V < 2 || m->emb_dim < 1) return TW_ERR_ARG;
   if (m->blank < 0 || m->blank >= m->V) return TW_ERR_ARG;
+  if (m->joiner_act != TW_ACT_TANH && m->joiner_act != TW_ACT_RELU) return TW_ERR_ARG;
   if (c->N < 1 || c->N > TW_MAX_BEAM || c->S < 1 || c->S > TW_MAX_SEGMENT) return TW_ERR_ARG;
   if (m->V - 1 < c->N) return TW_ERR_ARG;
   if (c->max_batch < 1 || c->max_T < 1 || c->max_iters_per_segment < 0 || c->max_tokens < 0) return TW_ERR_ARG;

@@ -8,7 +8,7 @@
 struct tw_handle {
   // model dimensions and search parameters
   int D_enc = 0, P = 0, J = 0, V = 0, blank = 0;
-  int pred_kind = 0, emb_dim = 0, L = 0, Hd = 0;
+  int pred_kind = 0, emb_dim = 0, L = 0, Hd = 0, joiner_act = 0;
   int N = 0, S = 0, mode = 0, max_batch = 0, max_T = 0, I_max = 0, U_cap = 0;
   int R_max = 0;
 

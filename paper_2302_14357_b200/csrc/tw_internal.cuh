@@ -59,6 +59,7 @@ struct JoinerRows {
   const int* row_slen;   // [R] valid frames (nullptr: S)
   const int* R_dev;      // device row count (nullptr: use R_max)
   int R_max, S, J, V;
+  int act;               // TW_ACT_TANH / TW_ACT_RELU
 };
 // z[(r,t), k] = sum_j tanh(E[e0[r]+t, j] + Pp[p[r], j]) * W_out[k, j] + b_out[k]; rows of padding
 // frames (t >= slen) are left untouched.

@@ -179,6 +179,7 @@ def _top1_agreement(cfg, S, batch, T):
     enc, lens = tw_synth.make_encoder_batch(cfg, batch)
     enc, lens = np.ascontiguousarray(enc[:, :T]), np.minimum(lens, T)
     dec = TwDecoder(weights_from_synth(m), N=cfg.N, S=S, mode=MODE_BF16, max_batch=batch, max_T=T)
+    assert dec.set_fused(True) == (cfg.V % 256 == 0)       # V = 501 runs the staged kernels
     tokens, olens, scores, status, rc = [x.cpu().numpy() if hasattr(x, "cpu") else x for x in dec.decode(enc, lens)]
     om = oracle_model(m)
     agree, gaps = 0, []
@@ -197,7 +198,7 @@ def test_decode_bf16_small_model_top1():
     assert rate >= 0.5 and gap < 0.5
 
 
-@pytest.mark.parametrize("name,S,batch,T", [("c1", 3, 4, 80), ("c3", 3, 2, 45)])
+@pytest.mark.parametrize("name,S,batch,T", [("c1", 3, 4, 80), ("c3", 3, 2, 45), ("p1", 3, 4, 60), ("p1", 5, 2, 50)])
 def test_decode_bf16_config_shapes_top1(name, S, batch, T):
     rate, gap, st = _top1_agreement(tw_synth.get_config(name), S, batch, T)
     print("%s bf16 top-1 agreement %.2f, max top-1 score gap %.3g" % (name, rate, gap))

@@ -92,6 +92,17 @@ def test_uniform_joiner_exact_ties():
     _run(cfg, 3, N=4, lengths=[7, 3, 6, 1, 2, 5], mutate=flat, max_iters=3)
 
 
+@pytest.mark.parametrize("S", [1, 3])
+def test_relu_joiner_small_model(S):
+    cfg = _tiny("lstm", 2, V=33, seed=14).with_(joiner_act="relu")
+    _run(cfg, S, lengths=[23, 6, 23, 1, 12, 19])
+
+
+def test_paper_shaped_relu_workload_subset():
+    """ReLU joiner, 3-layer LSTM predictor, 501-token vocabulary (not a multiple of 4)."""
+    _run(tw_synth.get_config("p1"), 3, batch=3, T=60)
+
+
 @pytest.mark.parametrize("S", [1, 2, 3, 5])
 def test_config1_subset(S):
     _run(tw_synth.get_config("c1"), S, batch=3, T=90)

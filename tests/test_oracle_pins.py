@@ -46,6 +46,27 @@ def test_joiner_closed_form_golden():
     np.testing.assert_allclose(out[0, 0], expected, atol=1e-14)
 
 
+def test_relu_joiner_closed_form_golden():
+    """The ReLU joiner of the paper's models on a hand-worked example; the negative pre-activation must
+    be clipped (tanh would give a different third decimal)."""
+    expected = np.array([r[0] for r in _read_golden("joiner_relu_closed_form.txt")])
+    model = rm.RnntModel(W_e=[[0.5], [0.2]], W_p=[[0.0], [-0.5]], W_out=[[2, 7], [0, 3], [4, 1]],
+                         b_out=[0, 0, 0], emb=np.zeros((3, 1)), activation="relu")
+    out = rm.joiner_log_probs(model, np.array([[1.0]]), np.array([[1.0]]))
+    np.testing.assert_allclose(out[0, 0], expected, atol=1e-14)
+    tanh_model = rm.RnntModel(W_e=[[0.5], [0.2]], W_p=[[0.0], [-0.5]], W_out=[[2, 7], [0, 3], [4, 1]],
+                              b_out=[0, 0, 0], emb=np.zeros((3, 1)))
+    assert np.abs(rm.joiner_log_probs(tanh_model, np.array([[1.0]]), np.array([[1.0]]))[0, 0] - expected).max() > 0.05
+
+
+def test_relu_model_unpruned_search_is_exact():
+    cfg, model, enc = tiny_case(V=4, T=4, pred="lstm", seed=31)
+    model.activation = "relu"
+    nbest, _ = tws.token_wise_beam_search(model, enc, N=400, S=3, max_len=2)
+    for y, s in nbest:
+        assert s == pytest.approx(ef.forward_log_prob(model, enc, y), abs=1e-11)
+
+
 def test_joiner_bias_and_broadcast_layout():
     """Output is [hypothesis, frame, vocab]; bias shifts one token's logit."""
     rng = np.random.default_rng(0)

@@ -22,6 +22,7 @@ class WorkloadConfig:
     S_values: Tuple[int, ...]   # segment sizes the workload sweeps
     dtype: str                  # "f32" | "bf16": storage precision of weights/inputs
     seed: int
+    joiner_act: str = "tanh"   # "tanh" | "relu"
 
     @property
     def P(self) -> int:
@@ -48,6 +49,10 @@ CONFIGS = {
     # throughput stress on the c3 model
     "c4": WorkloadConfig("c4", 512, 1000, (500, 1000), 1024, "lstm", 1024, 2, 1024,
                          1024, 4096, 4.0, 10, (10,), "bf16", 2),
+    # shaped like the paper's Librispeech model (Sec. 4.1): ReLU joiner, 500 sub-word units + blank,
+    # 3-layer LSTM predictor; the vocabulary is not a multiple of anything
+    "p1": WorkloadConfig("p1", 32, 300, (150, 300), 512, "lstm", 512, 3, 512,
+                         512, 501, 4.0, 5, (1, 3, 5), "bf16", 3, "relu"),
 }
 
 
