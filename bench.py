@@ -38,6 +38,7 @@ def parse_args():
     ap.add_argument("--mode", default="auto", choices=["auto", "f32", "bf16"])
     ap.add_argument("--batch", type=int, default=0, help="utterances per GPU (0: the workload's batch)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-lanes", action="store_true", help="decode the batch in one piece instead of two concurrent halves")
     ap.add_argument("--no-fused", action="store_true", help="bf16 mode: staged joiner kernels instead of the fused one")
     ap.add_argument("--cpu-frames", type=int, default=0, help="frames of the CPU-baseline sample (0: auto)")
     return ap.parse_args()
@@ -201,6 +202,8 @@ def run_ours(args, cfg, S):
     dec = TwDecoder(weights_from_synth(model), N=cfg.N, S=S, mode=mode, max_batch=B, max_T=cfg.T, joiner_act=cfg.joiner_act)
     if args.no_fused:
         dec.set_fused(False)
+    if args.no_lanes:
+        dec.set_lanes(False)
     enc = torch.from_numpy(enc_np).cuda()
     lens = torch.from_numpy(len_np).cuda()
     frames = int(len_np.sum())

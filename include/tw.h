@@ -250,6 +250,12 @@ int tw_set_fused(tw_handle* h, int on);
  * kernels one by one on `stream` instead (as it also does while profiling is on).  Default: on. */
 int tw_set_graph(tw_handle* h, int on);
 
+/* A handle with max_batch >= 256 also holds two internal decoders for half the batch each; tw_decode then
+ * splits a batch of 256 or more utterances in two halves and advances them concurrently on two streams
+ * (utterances are independent), which overlaps one half's small kernels with the other half's GEMMs.
+ * tw_set_lanes(h, 0) decodes the batch in one piece.  Default: on.  Off while profiling is on. */
+int tw_set_lanes(tw_handle* h, int on);
+
 /* Per-stage device timing of tw_decode with CUDA events on the decode stream (adds two event records
  * per stage per step); off by default. */
 int tw_set_profiling(tw_handle* h, int on);

@@ -12,7 +12,7 @@ TW_OK, TW_ERR_ARG, TW_ERR_ALLOC, TW_ERR_CUDA, TW_ERR_LIMIT, TW_ERR_STATE, TW_ERR
 
 EXPORTED_SYMBOLS = [
     "tw_init", "tw_destroy", "tw_decode", "tw_decode_host", "tw_max_tokens", "tw_project_encoder",
-    "tw_joiner_segment", "tw_expand", "tw_joiner_expand", "tw_predictor_step", "tw_get_stats", "tw_set_profiling", "tw_set_fused", "tw_set_graph",
+    "tw_joiner_segment", "tw_expand", "tw_joiner_expand", "tw_predictor_step", "tw_get_stats", "tw_set_profiling", "tw_set_fused", "tw_set_graph", "tw_set_lanes",
     "tw_joiner_expand_noalloc",
     "tw_last_cuda_error", "tw_strerror",
 ]
@@ -71,6 +71,7 @@ def load_library() -> C.CDLL:
     lib.tw_set_profiling.argtypes = [vp, C.c_int]
     lib.tw_set_fused.argtypes = [vp, C.c_int]
     lib.tw_set_graph.argtypes = [vp, C.c_int]
+    lib.tw_set_lanes.argtypes = [vp, C.c_int]
     lib.tw_joiner_expand_noalloc.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp]
     lib.tw_last_cuda_error.argtypes = [vp]
     lib.tw_strerror.argtypes = [C.c_int]
@@ -253,6 +254,9 @@ class TwDecoder:
 
     def set_graph(self, on: bool):
         self._check(self.lib.tw_set_graph(self.h, int(bool(on))), "tw_set_graph")
+
+    def set_lanes(self, on: bool):
+        self._check(self.lib.tw_set_lanes(self.h, int(bool(on))), "tw_set_lanes")
 
     def set_profiling(self, on: bool):
         self._check(self.lib.tw_set_profiling(self.h, int(bool(on))), "tw_set_profiling")

@@ -427,17 +427,33 @@ int tw_init(const tw_model* m, const tw_config* c, tw_handle** out) {
   if (!h) return TW_ERR_ALLOC;
   int s = init_impl(h, m, c);
   if (s != TW_OK) { tw_destroy(h); return s; }
+  // two lanes of half the batch each (tw_decode overlaps them); a failure here only disables lanes
+  if (c->max_batch >= 256) {
+    tw_config half = *c;
+    half.max_batch = (c->max_batch + 1) / 2;
+    for (int k = 0; k < 2; ++k) {
+      tw_handle* l = new (std::nothrow) tw_handle();
+      if (!l) break;
+      l->is_lane = true;
+      if (init_impl(l, m, &half) != TW_OK) { tw_destroy(l); break; }
+      h->lane[k] = l;
+    }
+    if (!h->lane[1] && h->lane[0]) { tw_destroy(h->lane[0]); h->lane[0] = nullptr; }
+  }
   *out = h;
   return TW_OK;
 }
 
 int tw_destroy(tw_handle* h) {
   if (!h) return TW_ERR_ARG;
+  for (int k = 0; k < 2; ++k)
+    if (h->lane[k]) { tw_destroy(h->lane[k]); h->lane[k] = nullptr; }
   cudaDeviceSynchronize();
   for (void* p : h->dev_allocs) cudaFree(p);
   for (cudaEvent_t e : h->events) cudaEventDestroy(e);
   if (h->graph_exec) cudaGraphExecDestroy(h->graph_exec);
   if (h->ev_order) cudaEventDestroy(h->ev_order);
+  if (h->ev_poll) cudaEventDestroy(h->ev_poll);
   if (h->own_stream) cudaStreamDestroy(h->own_stream);
   if (h->host_flag) cudaFreeHost(h->host_flag);
   delete h;
@@ -451,6 +467,12 @@ int tw_set_fused(tw_handle* h, int on) {
   if (!h) return TW_ERR_ARG;
   if (on && !h->bf.fused_ok) return TW_ERR_STATE;
   h->bf.fused_on = on != 0;
+  return TW_OK;
+}
+
+int tw_set_lanes(tw_handle* h, int on) {
+  if (!h) return TW_ERR_ARG;
+  h->lanes_on = on != 0;
   return TW_OK;
 }
 

@@ -56,6 +56,21 @@ struct tw_handle {
   cudaEvent_t ev_order = nullptr;
   cudaGraphExec_t graph_exec = nullptr;
   int graph_B = -1, graph_T = -1, graph_fused = -1, graph_launches = 0;
+  cudaEvent_t ev_poll = nullptr;
+
+  // state of the decode in flight (decode_begin .. decode_end)
+  struct Run {
+    int B = 0, T = 0;
+    int32_t* out_tokens = nullptr; int32_t* out_lens = nullptr; double* out_scores = nullptr; int32_t* out_status = nullptr;
+    cudaStream_t st = nullptr;
+    bool use_graph = false, active = false;
+    long long issued = 0, max_steps = 0;
+    int launches = 0;
+  } run;
+
+  // two internal decoders for half of max_batch each (see tw_decode); null for small handles
+  tw_handle* lane[2] = {nullptr, nullptr};
+  bool lanes_on = true, is_lane = false;
 
   // optional per-stage timing of tw_decode (tw_set_profiling): pooled events and the stage each closes
   bool profiling = false;

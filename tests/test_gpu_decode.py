@@ -121,6 +121,35 @@ def test_config4_shape_subset():
     _run(tw_synth.get_config("c4"), 10, batch=3, T=40, lengths=[40, 25, 33])
 
 
+@pytest.mark.parametrize("mode", [0, 1])
+def test_two_lanes_give_the_single_lane_result(mode):
+    """A large batch decoded as two concurrent halves (the default from 256 utterances up) equals the
+    batch decoded in one piece: utterances never interact."""
+    from paper_2302_14357_b200.binding import TwDecoder, weights_from_synth
+    cfg = tw_synth.WorkloadConfig("lanes", 300, 24, (0, 24), 64, "lstm", 64, 1, 64, 64, 256, 3.0, 3, (3,), "bf16", 9)
+    m = tw_synth.make_model(cfg)
+    enc, lens = tw_synth.make_encoder_batch(cfg)
+    dec = TwDecoder(weights_from_synth(m), N=cfg.N, S=3, mode=mode, max_batch=300, max_T=24)
+    a = [x.cpu().numpy() for x in dec.decode(enc, lens)[:4]]
+    sa = dec.stats()
+    dec.set_lanes(False)
+    b = [x.cpu().numpy() for x in dec.decode(enc, lens)[:4]]
+    sb = dec.stats()
+    for x, y in zip(a, b):
+        np.testing.assert_array_equal(x, y)
+    for key in ("frames", "calls", "joins", "rows", "limit_hits"):
+        assert sa[key] == sb[key], key
+    # an odd batch, and one below the lane threshold
+    dec.set_lanes(True)
+    c = [x.cpu().numpy() for x in dec.decode(enc[:257], lens[:257])[:4]]
+    d = [x.cpu().numpy() for x in dec.decode(enc[:5], lens[:5])[:4]]
+    for x, y in zip(c, a):
+        np.testing.assert_array_equal(x, y[:257])
+    for x, y in zip(d, a):
+        np.testing.assert_array_equal(x, y[:5])
+    dec.close()
+
+
 def test_decode_host_equals_device_decode():
     from paper_2302_14357_b200.binding import TwDecoder, weights_from_synth
     cfg = tw_synth.get_config("c0")
