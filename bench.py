@@ -101,7 +101,7 @@ def oracle_sample(cfg, S, frames, utt=0):
 def auto_cpu_frames(cfg):
     # sized for roughly 10-30 s of oracle time on a few host cores
     cost = cfg.J * cfg.V * cfg.N / (640 * 1024 * 10)
-    return int(max(24, min(cfg.T, 400 / max(cost, 0.05))))
+    return int(max(24, min(cfg.T, 600, 4000 / max(cost, 0.05))))
 
 
 def run_reference(args, cfg, S):

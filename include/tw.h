@@ -145,6 +145,28 @@ int tw_decode_host(tw_handle* h, const float* host_enc, const int32_t* host_leng
                    int32_t T, int32_t* host_out_tokens, int32_t* host_out_lens,
                    double* host_out_scores, int32_t* host_out_status, void* stream);
 
+/*
+ * Streaming (Sec. 3.2: the encoder output may arrive segment by segment, and the chunk size used for
+ * the encoder need not equal the decoding segment size S).  One session per handle at a time; the beam
+ * state (list B, hypotheses, predictor states) stays on the device between calls.
+ *   tw_stream_open   starts a session of B utterances with no frames.
+ *   tw_stream_push   appends chunk_lens[b] <= Tc frames of enc_chunk [B, Tc, D_enc] to utterance b and
+ *                    decodes every whole segment of S frames that is now available; frames short of a
+ *                    segment wait for the next push.  At most max_T frames per utterance in total
+ *                    (more are dropped and the utterance reports TW_ERR_LIMIT).
+ *   tw_stream_nbest  the current N best of every utterance (outputs as in tw_decode).
+ *   tw_stream_close  decodes the frames short of a segment as a last, shorter one and returns the final
+ *                    N best; tw_get_stats then covers the whole session.
+ * After tw_stream_close the result is exactly that of tw_decode on the concatenated frames.
+ * All four synchronise before returning.  TW_ERR_STATE without an open session.
+ */
+int tw_stream_open(tw_handle* h, int32_t B, void* stream);
+int tw_stream_push(tw_handle* h, const float* enc_chunk, const int32_t* chunk_lens, int32_t Tc, void* stream);
+int tw_stream_nbest(tw_handle* h, int32_t* out_tokens, int32_t* out_lens, double* out_scores,
+                    int32_t* out_status, void* stream);
+int tw_stream_close(tw_handle* h, int32_t* out_tokens, int32_t* out_lens, double* out_scores,
+                    int32_t* out_status, void* stream);
+
 /* U_cap of this handle (row length of out_tokens). */
 int tw_max_tokens(const tw_handle* h);
 

@@ -13,6 +13,7 @@ TW_OK, TW_ERR_ARG, TW_ERR_ALLOC, TW_ERR_CUDA, TW_ERR_LIMIT, TW_ERR_STATE, TW_ERR
 EXPORTED_SYMBOLS = [
     "tw_init", "tw_destroy", "tw_decode", "tw_decode_host", "tw_max_tokens", "tw_project_encoder",
     "tw_joiner_segment", "tw_expand", "tw_joiner_expand", "tw_predictor_step", "tw_get_stats", "tw_set_profiling", "tw_set_fused", "tw_set_graph", "tw_set_lanes",
+    "tw_stream_open", "tw_stream_push", "tw_stream_nbest", "tw_stream_close",
     "tw_joiner_expand_noalloc",
     "tw_last_cuda_error", "tw_strerror",
 ]
@@ -72,6 +73,10 @@ def load_library() -> C.CDLL:
     lib.tw_set_fused.argtypes = [vp, C.c_int]
     lib.tw_set_graph.argtypes = [vp, C.c_int]
     lib.tw_set_lanes.argtypes = [vp, C.c_int]
+    lib.tw_stream_open.argtypes = [vp, i32, vp]
+    lib.tw_stream_push.argtypes = [vp, vp, vp, i32, vp]
+    lib.tw_stream_nbest.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.tw_stream_close.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.tw_joiner_expand_noalloc.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp]
     lib.tw_last_cuda_error.argtypes = [vp]
     lib.tw_strerror.argtypes = [C.c_int]
@@ -197,6 +202,34 @@ class TwDecoder:
                                      lens.ctypes.data, scores.ctypes.data, status.ctypes.data, self._stream())
         self._check(rc, "tw_decode_host", allow_limit=True)
         return tokens, lens, scores, status, rc
+
+    def _nbest_buffers(self, B):
+        torch = self._torch
+        return (torch.empty((B, self.N, self.U_cap), dtype=torch.int32, device=self.device),
+                torch.empty((B, self.N), dtype=torch.int32, device=self.device),
+                torch.empty((B, self.N), dtype=torch.float64, device=self.device),
+                torch.empty((B,), dtype=torch.int32, device=self.device))
+
+    def stream_open(self, B: int):
+        self._check(self.lib.tw_stream_open(self.h, B, self._stream()), "tw_stream_open")
+        self._stream_B = B
+
+    def stream_push(self, enc_chunk, chunk_lens):
+        """tw_stream_push: enc_chunk [B, Tc, D_enc], chunk_lens [B] valid frames of the chunk per utterance."""
+        enc_chunk, chunk_lens = self._f32(enc_chunk), self._i32(chunk_lens)
+        self._check(self.lib.tw_stream_push(self.h, enc_chunk.data_ptr(), chunk_lens.data_ptr(), enc_chunk.shape[1],
+                                            self._stream()), "tw_stream_push", allow_limit=True)
+
+    def stream_nbest(self):
+        out = self._nbest_buffers(self._stream_B)
+        self._check(self.lib.tw_stream_nbest(self.h, *[t.data_ptr() for t in out], self._stream()), "tw_stream_nbest")
+        return out
+
+    def stream_close(self):
+        out = self._nbest_buffers(self._stream_B)
+        rc = self.lib.tw_stream_close(self.h, *[t.data_ptr() for t in out], self._stream())
+        self._check(rc, "tw_stream_close", allow_limit=True)
+        return out + (rc,)
 
     def project_encoder(self, enc):
         enc = self._f32(enc).reshape(-1, self.D_enc)

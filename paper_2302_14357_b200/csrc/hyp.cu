@@ -65,7 +65,7 @@ __global__ void __launch_bounds__(kThreads) hyp_init_kernel(HypState hs, const i
     int len = lengths[b], st = TW_OK;
     if (len < 0) { len = 0; st = TW_ERR_ARG; }
     if (len > T) { len = T; st = TW_ERR_ARG; }
-    hs.len[b] = len; hs.status[b] = st;
+    hs.len[b] = len; hs.status[b] = st; hs.avail[b] = len;
     hs.calls[b] = 0; hs.joins[b] = 0; hs.iters[b] = 0; hs.cursor[b] = 0; hs.n_new[b] = 0;
     hs.t0[b] = 0; hs.slen[b] = 0; hs.nA[b] = 0;
     hs.slot_len[gs] = 0; hs.slot_hash[gs] = kHashSeed;
@@ -359,6 +359,32 @@ __global__ void __launch_bounds__(1024) compact_kernel(HypState hs, int B, int T
   }
 }
 
+__global__ void stream_rows_kernel(HypState hs, const int* chunk_lens, int B, int Tc, int max_T, int dump_row, int* oidx) {
+  const int m = blockIdx.x * blockDim.x + threadIdx.x;
+  if (m >= B * Tc) return;
+  const int b = m / Tc, i = m - b * Tc;
+  const int have = hs.avail[b];
+  const bool ok = i < chunk_lens[b] && have + i < max_T;
+  oidx[m] = ok ? b * max_T + have + i : dump_row;
+}
+
+__global__ void __launch_bounds__(kThreads) stream_advance_kernel(HypState hs, const int* chunk_lens, int max_T, int closing) {
+  const int b = blockIdx.x;
+  __shared__ int s_go;
+  if (threadIdx.x == 0) {
+    int add = chunk_lens ? max(chunk_lens[b], 0) : 0;
+    int have = hs.avail[b];
+    if (have + add > max_T) { add = max_T - have; hs.status[b] = TW_ERR_LIMIT; }
+    have += add;
+    hs.avail[b] = have;
+    const int len = closing ? have : (have / hs.S) * hs.S;    // only whole segments while the stream is open
+    hs.len[b] = len;
+    s_go = (hs.nA[b] == 0 && hs.t0[b] + hs.slen[b] < len);
+  }
+  __syncthreads();
+  if (s_go) turn_over(hs, b);
+}
+
 // ChooseNBest(B) at the end of the utterance, best first.
 __global__ void __launch_bounds__(kThreads) finish_kernel(HypState hs, int* out_tokens, int* out_lens,
                                                           double* out_scores, int* out_status) {
@@ -413,6 +439,15 @@ void launch_hyp_step(const HypState& hs, int B, cudaStream_t st) {
 }
 void launch_compact(const HypState& hs, int B, int T, cudaStream_t st) {
   compact_kernel<<<1, 1024, 0, st>>>(hs, B, T);
+}
+void launch_stream_rows(const HypState& hs, const int* chunk_lens, int B, int Tc, int max_T, int dump_row,
+                        int* oidx, cudaStream_t st) {
+  const int n = B * Tc;
+  if (n > 0) stream_rows_kernel<<<(n + 255) / 256, 256, 0, st>>>(hs, chunk_lens, B, Tc, max_T, dump_row, oidx);
+}
+void launch_stream_advance(const HypState& hs, const int* chunk_lens, int B, int max_T, int closing,
+                           cudaStream_t st) {
+  if (B > 0) stream_advance_kernel<<<B, kThreads, 0, st>>>(hs, chunk_lens, max_T, closing);
 }
 void launch_finish(const HypState& hs, int B, int* out_tokens, int* out_lens, double* out_scores,
                    int* out_status, cudaStream_t st) {

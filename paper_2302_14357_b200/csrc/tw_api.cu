@@ -230,7 +230,7 @@ int build_workspace(tw_handle* h) {
   hs.stateless = (h->pred_kind == TW_PRED_STATELESS);
   const size_t nb = (size_t)B, nslot = nb * hs.capSlot, nB = nb * hs.capB, R = (size_t)h->R_max;
   int** per_utt[] = {&hs.len, &hs.t0, &hs.slen, &hs.nA, &hs.nB, &hs.nTop, &hs.iters, &hs.status,
-                     &hs.cursor, &hs.n_new, &hs.calls, &hs.joins, &hs.row_off, &hs.new_off};
+                     &hs.cursor, &hs.n_new, &hs.calls, &hs.joins, &hs.row_off, &hs.new_off, &hs.avail};
   for (int** p : per_utt) TW_TRY(dev_alloc(h, p, nb));
   TW_TRY(dev_alloc(h, &hs.A_slot, nb * kMaxBeam));
   TW_TRY(dev_alloc(h, &hs.A_ls, nb * kMaxBeam));
@@ -272,7 +272,10 @@ int build_workspace(tw_handle* h) {
   TW_TRY(dev_alloc(h, &hs.la_d, R * S));
   TW_TRY(dev_alloc(h, &hs.ldnb, R * h->V));
   TW_TRY(dev_alloc(h, &hs.logp, R * S * h->V));
-  TW_TRY(dev_alloc(h, &h->E, nb * h->max_T * h->J));
+  TW_TRY(dev_alloc(h, &h->E, (nb * h->max_T + 1) * h->J));   // + one dump row for frames a streamed chunk does not hold
+  TW_TRY(dev_alloc(h, &h->stream_oidx, nb * h->max_T));
+  TW_TRY(dev_alloc(h, &h->zero_len, nb));
+  TW_CUDA(h, cudaMemset(h->zero_len, 0, nb * sizeof(int)));
   TW_CUDA(h, cudaMemset(hs.scalars, 0, kScCount * sizeof(int)));
   TW_CUDA(h, cudaMemset(hs.rows_total, 0, 2 * sizeof(long long)));
   TW_CUDA(h, cudaHostAlloc((void**)&h->host_flag, (kScCount + 4) * sizeof(long long), cudaHostAllocDefault));
@@ -513,3 +516,4 @@ const char* tw_strerror(int s) {
 
 #include "tw_api_stages.inc"
 #include "tw_api_decode.inc"
+#include "tw_api_stream.inc"

@@ -24,6 +24,9 @@ struct tw_handle {
   float* E = nullptr;         // projected encoder frames [max_batch * max_T, J]
   float* gates = nullptr;     // LSTM gate pre-activations [R_max, 4 Hd]
   int *stage_e0 = nullptr, *stage_slen = nullptr;   // [R_max] scratch of the stage entry points
+  int* stream_oidx = nullptr;   // [max_batch * max_T] destination rows of a pushed chunk's frames
+  int* zero_len = nullptr;      // [max_batch] zeros
+  int stream_B = 0;             // utterances of the open streaming session (0: none)
 
   // TW_MODE_BF16: bf16 copies of the GEMM operands with their tensor maps
   struct {

@@ -108,6 +108,7 @@ struct HypState {
   int stateless;
   // per utterance [B]
   int *len, *t0, *slen, *nA, *nB, *nTop, *iters, *status, *cursor, *n_new, *calls, *joins;
+  int* avail;    // streaming: frames pushed so far (len is the part of them that may be decoded now)
   // list A: [B][kMaxBeam]
   int* A_slot; double* A_ls; double* A_ld;   // A_ld [B][kMaxBeam][S]
   // list B of Algorithm 1 (hypotheses finished for this segment): [B][capB]
@@ -139,6 +140,14 @@ struct HypState {
 void launch_hyp_init(const HypState& hs, const int* lengths, int B, int T, cudaStream_t st);
 void launch_hyp_step(const HypState& hs, int B, cudaStream_t st);
 void launch_compact(const HypState& hs, int B, int T, cudaStream_t st);
+// Streaming.  stream_rows: destination row in E of every frame of a pushed chunk [B, Tc] (frames past
+// chunk_lens[b] or past max_T go to `dump_row`); stream_advance: avail += chunk_lens (clamped to max_T,
+// flagging TW_ERR_LIMIT), len = whole segments of avail (all of avail when closing), and a turn-over
+// for every utterance that was waiting for frames.
+void launch_stream_rows(const HypState& hs, const int* chunk_lens, int B, int Tc, int max_T, int dump_row,
+                        int* oidx, cudaStream_t st);
+void launch_stream_advance(const HypState& hs, const int* chunk_lens, int B, int max_T, int closing,
+                           cudaStream_t st);
 void launch_finish(const HypState& hs, int B, int* out_tokens, int* out_lens, double* out_scores,
                    int* out_status, cudaStream_t st);
 
