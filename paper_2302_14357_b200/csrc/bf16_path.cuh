@@ -42,12 +42,19 @@ int gemm_bf16_setup();
 void launch_gemm_bf16(const CUtensorMap& tmA, const CUtensorMap& tmB128, const CUtensorMap& tmB256,
                       const GemmBf16Params& p, cudaStream_t st);
 
+// LSTM gate GEMM (epi == 1) as a single wave of one tile per CTA when 128 x 256 tiles would need a second,
+// nearly empty wave; returns false (nothing launched) when the shape does not call for it.
+// tmB64 / tmB32: maps of B with 64- and 32-row boxes
+bool launch_gemm_lstm_wide(const CUtensorMap& tmA, const CUtensorMap& tmB64, const CUtensorMap& tmB32,
+                           const GemmBf16Params& p, cudaStream_t st);
+
 // A bf16 matrix with its tensor maps
 struct Bf16Mat {
   __nv_bfloat16* ptr = nullptr;
   long long rows = 0, K = 0;
   CUtensorMap as_A;            // box 128 rows
   CUtensorMap as_B128, as_B256;
+  CUtensorMap as_B64, as_B32;
 };
 
 // elementwise helpers ---------------------------------------------------------------------------

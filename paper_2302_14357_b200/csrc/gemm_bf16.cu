@@ -26,6 +26,7 @@ struct Cfg {
 };
 
 __device__ __forceinline__ float sigmoid_fast(float x) { return __fdividef(1.f, 1.f + __expf(-x)); }
+
 __device__ __forceinline__ float tanh_fast_g(float x) {
   float y;
   asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -207,6 +208,165 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   if (warp == 1) tmem_dealloc(tmem_base, 2 * BN);
 }
 
+// ---- single-wave LSTM gate GEMM ------------------------------------------------------------------
+// For a handful of row tiles and a wide N (the gate GEMMs of a step: some 10 row tiles x 4 Hd columns)
+// 128 x 256 tiles need a second, almost empty wave.  Here the columns of a row tile are split evenly
+// over floor(#SM / row tiles) CTAs in units of 32 columns, so every CTA owns exactly one tile of up to
+// 320 columns (one tcgen05.mma of N <= 256 plus one of N <= 64 per K step, accumulators side by side in
+// TMEM) and the whole GEMM is one wave.  B is loaded in boxes of 64 (and one of 32) rows.
+constexpr int kWideMaxBN = 320, kWideStages = 4, kWideEpiWarps = 16;
+constexpr int kThreadsWide = 64 + 32 * kWideEpiWarps;
+constexpr uint32_t kWideABytes = BM * BK * 2, kWideBBytes = kWideMaxBN * BK * 2;
+constexpr size_t kWideSmem = (size_t)kWideStages * (kWideABytes + kWideBBytes) + 1024 + 256;
+
+__global__ void __launch_bounds__(kThreadsWide, 1)
+gemm_lstm_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB64,
+                      const __grid_constant__ CUtensorMap tmB32, GemmBf16Params p, int n_split) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* sA = smem;
+  uint8_t* sB = smem + kWideStages * kWideABytes;
+  uint64_t* full = reinterpret_cast<uint64_t*>(sB + kWideStages * kWideBBytes);
+  uint64_t* empty = full + kWideStages;
+  uint64_t* acc_full = empty + kWideStages;
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(acc_full + 1);
+
+  const int M = p.M_dev ? *p.M_dev : p.M;
+  const int mt = blockIdx.x / n_split, ns = blockIdx.x - mt * n_split;
+  const int m0 = mt * BM;
+  if (m0 >= M) return;                                   // the whole CTA, before any barrier exists
+  const int units = p.N >> 5, ubase = units / n_split, urem = units - ubase * n_split;
+  const int u0 = ns * ubase + (ns < urem ? ns : urem), nu = ubase + (ns < urem ? 1 : 0);
+  if (nu == 0) return;
+  const int n0 = u0 * 32, w = nu * 32;                   // this CTA's columns [n0, n0 + w), w <= kWideMaxBN
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int num_kb = (p.K + BK - 1) / BK;
+
+  if (threadIdx.x == 0) {
+    prefetch_tensormap(&tmA);
+    prefetch_tensormap(&tmB64);
+    prefetch_tensormap(&tmB32);
+    for (int s = 0; s < kWideStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(acc_full, 1);
+    fence_barrier_init();
+    fence_proxy_async_smem();
+  }
+  if (warp == 1) { tmem_alloc(tmem_holder, 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_holder;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      for (int kb = 0; kb < num_kb; ++kb) {
+        const int s = kb % kWideStages;
+        const uint32_t ph = (kb / kWideStages) & 1;
+        if (!mbar_wait(&empty[s], ph ^ 1, p.err)) break;
+        mbar_expect_tx(&full[s], kWideABytes + (uint32_t)w * (BK * 2));
+        tma_load_2d(sA + s * kWideABytes, &tmA, &full[s], kb * BK, m0);
+        uint8_t* bdst = sB + s * kWideBBytes;
+        int r = 0;
+        for (; r + 64 <= w; r += 64) tma_load_2d(bdst + r * (BK * 2), &tmB64, &full[s], kb * BK, n0 + r);
+        if (r < w) tma_load_2d(bdst + r * (BK * 2), &tmB32, &full[s], kb * BK, n0 + r);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const int n1 = w < 256 ? w : 256, n2 = w - n1;
+      const uint32_t idesc1 = make_idesc_bf16(BM, n1), idesc2 = make_idesc_bf16(BM, n2);
+      bool ok = true;
+      for (int kb = 0; kb < num_kb; ++kb) {
+        const int s = kb % kWideStages;
+        const uint32_t ph = (kb / kWideStages) & 1;
+        ok = mbar_wait(&full[s], ph, p.err);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t a_addr = smem_u32(sA + s * kWideABytes), b_addr = smem_u32(sB + s * kWideBBytes);
+#pragma unroll
+        for (int k = 0; k < BK / 16; ++k) {
+          const uint64_t da = make_desc_k_sw128(a_addr + k * 32);
+          umma_bf16(tmem_base, da, make_desc_k_sw128(b_addr + k * 32), idesc1, (kb | k) != 0);
+          if (n2 > 0)
+            umma_bf16(tmem_base + 256u, da, make_desc_k_sw128(b_addr + 256 * (BK * 2) + k * 32), idesc2, (kb | k) != 0);
+        }
+        umma_commit(&empty[s]);
+      }
+      if (ok) umma_commit(acc_full);
+    }
+  } else {
+    // Epilogue: the LSTM cell, a row per thread; warp group grp takes the 32-column chunks grp, grp + 4, grp + 8.
+    const int ew = warp - 2, q = warp & 3, grp = ew >> 2;
+    const int m = m0 + q * 32 + lane;
+    const bool live = m < M;                                   // tcgen05.ld below is warp-wide: idle rows stay in the loop
+    const long long stride = (long long)p.lstm.L * 2 * p.lstm.Hd, lo = (long long)p.lstm.l * 2 * p.lstm.Hd;
+    const float* cin = nullptr;
+    const float* arow = nullptr;
+    float* hout = nullptr;
+    __nv_bfloat16* xrow = nullptr;
+    if (live) {
+      cin = p.lstm.hc_in + (long long)(p.lstm.idx_in ? p.lstm.idx_in[m] : m) * stride + lo + p.lstm.Hd;
+      hout = p.lstm.hc_out + (long long)(p.lstm.idx_out ? p.lstm.idx_out[m] : m) * stride + lo;
+      xrow = p.lstm.xnext + (long long)m * p.lstm.ld_xnext;
+      if (p.addend) arow = p.addend + (long long)(p.add_idx ? p.add_idx[m] : m) * p.ld_add;
+      // while the contraction runs: pull this thread's epilogue inputs (table row segments, parent's c) into L2
+      for (int c = grp; c < nu; c += kWideEpiWarps / 4) {
+        if (arow) prefetch_l2(arow + n0 + c * 32);
+        prefetch_l2(cin + ((n0 + c * 32) >> 2));
+      }
+    }
+    bool ok = mbar_wait(acc_full, 0, p.err);
+    ok = __all_sync(0xffffffffu, ok);
+    if (ok) {
+      tc_fence_after();
+#pragma unroll 1
+      for (int c = grp; c < nu; c += kWideEpiWarps / 4) {
+        float v[32];
+        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), v);
+        if (!live) continue;
+        const int nb = n0 + c * 32, j0 = nb >> 2;              // 8 whole hidden units (gate columns interleaved)
+        if (p.bias) {
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {
+            const float4 b4 = __ldg(reinterpret_cast<const float4*>(p.bias + nb + j));
+            v[j] += b4.x; v[j + 1] += b4.y; v[j + 2] += b4.z; v[j + 3] += b4.w;
+          }
+        }
+        if (arow) {
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {
+            const float4 a4 = __ldg(reinterpret_cast<const float4*>(arow + nb + j));
+            v[j] += a4.x; v[j + 1] += a4.y; v[j + 2] += a4.z; v[j + 3] += a4.w;
+          }
+        }
+        const float4 c0 = *reinterpret_cast<const float4*>(cin + j0), c1 = *reinterpret_cast<const float4*>(cin + j0 + 4);
+        const float cp[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+        float hn[8], cn[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const float cc = sigmoid_fast(v[4 * u + 1]) * cp[u] + sigmoid_fast(v[4 * u]) * tanh_fast_g(v[4 * u + 2]);
+          cn[u] = cc;
+          hn[u] = sigmoid_fast(v[4 * u + 3]) * tanh_fast_g(cc);
+        }
+        float* cout = hout + p.lstm.Hd;
+        *reinterpret_cast<float4*>(hout + j0) = make_float4(hn[0], hn[1], hn[2], hn[3]);
+        *reinterpret_cast<float4*>(hout + j0 + 4) = make_float4(hn[4], hn[5], hn[6], hn[7]);
+        *reinterpret_cast<float4*>(cout + j0) = make_float4(cn[0], cn[1], cn[2], cn[3]);
+        *reinterpret_cast<float4*>(cout + j0 + 4) = make_float4(cn[4], cn[5], cn[6], cn[7]);
+        __nv_bfloat162 b0 = __floats2bfloat162_rn(hn[0], hn[1]), b1 = __floats2bfloat162_rn(hn[2], hn[3]);
+        __nv_bfloat162 b2 = __floats2bfloat162_rn(hn[4], hn[5]), b3 = __floats2bfloat162_rn(hn[6], hn[7]);
+        uint4 pk;
+        pk.x = *reinterpret_cast<uint32_t*>(&b0); pk.y = *reinterpret_cast<uint32_t*>(&b1);
+        pk.z = *reinterpret_cast<uint32_t*>(&b2); pk.w = *reinterpret_cast<uint32_t*>(&b3);
+        *reinterpret_cast<uint4*>(xrow + j0) = pk;
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem_base, 512);
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -243,18 +403,38 @@ int gemm_bf16_setup() {
   cudaError_t e2 = cudaFuncSetAttribute(gemm_bf16_kernel<128, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<128>::kSmem);
   cudaError_t e3 = cudaFuncSetAttribute(gemm_bf16_kernel<256, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<256>::kSmem);
   cudaError_t e4 = cudaFuncSetAttribute(gemm_bf16_kernel<128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<128>::kSmem);
-  return (e1 == cudaSuccess && e2 == cudaSuccess && e3 == cudaSuccess && e4 == cudaSuccess) ? TW_OK : TW_ERR_CUDA;
+  cudaError_t e5 = cudaFuncSetAttribute(gemm_lstm_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kWideSmem);
+  return (e1 == cudaSuccess && e2 == cudaSuccess && e3 == cudaSuccess && e4 == cudaSuccess && e5 == cudaSuccess) ? TW_OK : TW_ERR_CUDA;
 }
 
-void launch_gemm_bf16(const CUtensorMap& tmA, const CUtensorMap& tmB128, const CUtensorMap& tmB256,
-                      const GemmBf16Params& p, cudaStream_t st) {
-  if (p.M <= 0 || p.N <= 0) return;
+static int sm_count() {
   static int num_sms = 0;
   if (num_sms == 0) {
     int dev = 0;
     cudaGetDevice(&dev);
     if (cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms <= 0) num_sms = 148;
   }
+  return num_sms;
+}
+
+bool launch_gemm_lstm_wide(const CUtensorMap& tmA, const CUtensorMap& tmB64, const CUtensorMap& tmB32,
+                           const GemmBf16Params& p, cudaStream_t st) {
+  if (p.epi != 1 || p.M <= 0 || p.N <= 0 || (p.N & 31) != 0) return false;
+  const int num_sms = sm_count();
+  const int mt = (p.M + BM - 1) / BM, nt256 = (p.N + 255) / 256;
+  if ((long long)mt * nt256 <= num_sms) return false;          // 128 x 256 tiles are one wave already
+  const int n_split = num_sms / mt;
+  if (n_split < 1) return false;
+  const int units = p.N >> 5;
+  if (((units + n_split - 1) / n_split) * 32 > kWideMaxBN) return false;
+  gemm_lstm_wide_kernel<<<mt * n_split, kThreadsWide, kWideSmem, st>>>(tmA, tmB64, tmB32, p, n_split);
+  return true;
+}
+
+void launch_gemm_bf16(const CUtensorMap& tmA, const CUtensorMap& tmB128, const CUtensorMap& tmB256,
+                      const GemmBf16Params& p, cudaStream_t st) {
+  if (p.M <= 0 || p.N <= 0) return;
+  const int num_sms = sm_count();
   const int mt = (p.M + BM - 1) / BM;
   const int nt256 = (p.N + 255) / 256, nt128 = (p.N + 127) / 128;
   // small problems: narrower tiles put more SMs to work
