@@ -31,6 +31,8 @@ __global__ void gather_concat_bf16_kernel(const float* __restrict__ src1, const 
 }
 
 __global__ void gather_parents_bf16_kernel(GatherParents g, const int* n_dev, int n_max) {
+  pdl_wait();
+  pdl_trigger();
   const int n = n_dev ? *n_dev : n_max;
   const int r = blockIdx.x, l = blockIdx.y;
   if (r >= n) return;
@@ -90,7 +92,7 @@ void launch_gather_concat_bf16(const float* src1, const int* idx1, long long ld1
 
 void launch_gather_parents_bf16(const GatherParents& g, const int* n_dev, int n_max, cudaStream_t st) {
   if (n_max <= 0 || g.L <= 0) return;
-  gather_parents_bf16_kernel<<<dim3(n_max, g.L), 128, 0, st>>>(g, n_dev, n_max);
+  launch_pdl(gather_parents_bf16_kernel, dim3(n_max, g.L), dim3(128), 0, st, g, n_dev, n_max);
 }
 
 void launch_permute_cols_f32(const float* src, const int* perm, long long rows, int cols, float* dst, cudaStream_t st) {

@@ -47,10 +47,6 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   uint64_t* acc_empty = acc_full + 2;          // [2]
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(acc_empty + 2);
 
-  const int M = p.M_dev ? *p.M_dev : p.M;
-  const int m_tiles = (M + BM - 1) / BM, n_tiles = (p.N + BN - 1) / BN;
-  const int num_tiles = m_tiles * n_tiles;
-  if ((int)blockIdx.x >= num_tiles) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_kb = (p.K + BK - 1) / BK;
 
@@ -67,6 +63,12 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_holder;
+  // the set-up above touched only this CTA: it may overlap the tail of the kernel that produces A and M
+  pdl_wait();
+  pdl_trigger();
+  const int M = p.M_dev ? *p.M_dev : p.M;
+  const int m_tiles = (M + BM - 1) / BM, n_tiles = (p.N + BN - 1) / BN;
+  const int num_tiles = m_tiles * n_tiles;     // a CTA past the last tile runs no loop iteration below
 
   if (warp == 0) {
     if (lane == 0) {
@@ -231,13 +233,10 @@ gemm_lstm_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
   uint64_t* acc_full = empty + kWideStages;
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(acc_full + 1);
 
-  const int M = p.M_dev ? *p.M_dev : p.M;
   const int mt = blockIdx.x / n_split, ns = blockIdx.x - mt * n_split;
   const int m0 = mt * BM;
-  if (m0 >= M) return;                                   // the whole CTA, before any barrier exists
   const int units = p.N >> 5, ubase = units / n_split, urem = units - ubase * n_split;
   const int u0 = ns * ubase + (ns < urem ? ns : urem), nu = ubase + (ns < urem ? 1 : 0);
-  if (nu == 0) return;
   const int n0 = u0 * 32, w = nu * 32;                   // this CTA's columns [n0, n0 + w), w <= kWideMaxBN
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_kb = (p.K + BK - 1) / BK;
@@ -256,8 +255,14 @@ gemm_lstm_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_holder;
+  // the set-up above touched only this CTA: it may overlap the tail of the kernel that produces A and M
+  pdl_wait();
+  pdl_trigger();
+  const int M = p.M_dev ? *p.M_dev : p.M;
+  const bool active = m0 < M && nu > 0;                  // an idle CTA skips the roles and only frees its TMEM
 
-  if (warp == 0) {
+  if (!active) {
+  } else if (warp == 0) {
     if (lane == 0) {
       for (int kb = 0; kb < num_kb; ++kb) {
         const int s = kb % kWideStages;
@@ -427,7 +432,7 @@ bool launch_gemm_lstm_wide(const CUtensorMap& tmA, const CUtensorMap& tmB64, con
   if (n_split < 1) return false;
   const int units = p.N >> 5;
   if (((units + n_split - 1) / n_split) * 32 > kWideMaxBN) return false;
-  gemm_lstm_wide_kernel<<<mt * n_split, kThreadsWide, kWideSmem, st>>>(tmA, tmB64, tmB32, p, n_split);
+  launch_pdl(gemm_lstm_wide_kernel, dim3(mt * n_split), dim3(kThreadsWide), kWideSmem, st, tmA, tmB64, tmB32, p, n_split);
   return true;
 }
 
@@ -440,13 +445,13 @@ void launch_gemm_bf16(const CUtensorMap& tmA, const CUtensorMap& tmB128, const C
   // small problems: narrower tiles put more SMs to work
   if ((long long)mt * nt256 >= num_sms) {
     const int grid = (int)((long long)mt * nt256 < num_sms ? mt * nt256 : num_sms);
-    if (p.epi == 1) gemm_bf16_kernel<256, 1><<<grid, kThreadsGemm, Cfg<256>::kSmem, st>>>(tmA, tmB256, p);
-    else gemm_bf16_kernel<256, 0><<<grid, kThreadsGemm, Cfg<256>::kSmem, st>>>(tmA, tmB256, p);
+    if (p.epi == 1) launch_pdl(gemm_bf16_kernel<256, 1>, dim3(grid), dim3(kThreadsGemm), Cfg<256>::kSmem, st, tmA, tmB256, p);
+    else launch_pdl(gemm_bf16_kernel<256, 0>, dim3(grid), dim3(kThreadsGemm), Cfg<256>::kSmem, st, tmA, tmB256, p);
   } else {
     const long long tiles = (long long)mt * nt128;
     const int grid = (int)(tiles < num_sms ? tiles : num_sms);
-    if (p.epi == 1) gemm_bf16_kernel<128, 1><<<grid, kThreadsGemm, Cfg<128>::kSmem, st>>>(tmA, tmB128, p);
-    else gemm_bf16_kernel<128, 0><<<grid, kThreadsGemm, Cfg<128>::kSmem, st>>>(tmA, tmB128, p);
+    if (p.epi == 1) launch_pdl(gemm_bf16_kernel<128, 1>, dim3(grid), dim3(kThreadsGemm), Cfg<128>::kSmem, st, tmA, tmB128, p);
+    else launch_pdl(gemm_bf16_kernel<128, 0>, dim3(grid), dim3(kThreadsGemm), Cfg<128>::kSmem, st, tmA, tmB128, p);
   }
 }
 

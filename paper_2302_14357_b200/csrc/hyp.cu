@@ -99,6 +99,8 @@ __global__ void __launch_bounds__(kStepThreads) hyp_step_kernel(HypState hs) {
   __shared__ int s_keep_h[kMaxBeam], s_keep_k[kMaxBeam], s_keep_slot[kMaxBeam];
   __shared__ double s_keep_ls[kMaxBeam];
 
+  pdl_wait();
+  pdl_trigger();
   const int b = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int H = hs.nA[b];
@@ -293,6 +295,8 @@ __global__ void __launch_bounds__(1024) compact_kernel(HypState hs, int B, int T
   __shared__ int s_a[1024], s_n[1024];
   __shared__ int s_base_a, s_base_n, s_frames;
   const int tid = threadIdx.x;
+  pdl_wait();
+  pdl_trigger();
   if (tid == 0) { s_base_a = 0; s_base_n = 0; s_frames = 0; }
   __syncthreads();
   // exclusive scans of the list sizes -> row_off, new_off
@@ -435,10 +439,10 @@ void launch_hyp_init(const HypState& hs, const int* lengths, int B, int T, cudaS
   if (B > 0) hyp_init_kernel<<<B, kThreads, 0, st>>>(hs, lengths, T);
 }
 void launch_hyp_step(const HypState& hs, int B, cudaStream_t st) {
-  if (B > 0) hyp_step_kernel<<<B, kStepThreads, 0, st>>>(hs);
+  if (B > 0) launch_pdl(hyp_step_kernel, dim3(B), dim3(kStepThreads), 0, st, hs);
 }
 void launch_compact(const HypState& hs, int B, int T, cudaStream_t st) {
-  compact_kernel<<<1, 1024, 0, st>>>(hs, B, T);
+  launch_pdl(compact_kernel, dim3(1), dim3(1024), 0, st, hs, B, T);
 }
 void launch_stream_rows(const HypState& hs, const int* chunk_lens, int B, int Tc, int max_T, int dump_row,
                         int* oidx, cudaStream_t st) {

@@ -47,6 +47,8 @@ __global__ void __launch_bounds__(kMaxT) scan_select_kernel(ScanSelectArgs a) {
   __shared__ int s_wk[kMaxT / 32][kMaxBeam];
   __shared__ int s_wn[kMaxT / 32];
 
+  pdl_wait();
+  pdl_trigger();
   const int R = a.R_dev ? *a.R_dev : a.R_max;
   const int r = blockIdx.x;
   if (r >= R) return;
@@ -249,8 +251,8 @@ void launch_scan_select(const ScanSelectArgs& a, bool fast_math, cudaStream_t st
   const size_t smem = a.dnb_in ? scan_select_smem_bytes(1, a.V) : scan_select_smem_bytes(a.S, a.V);
   // a row that takes most of an SM's shared memory runs alone there: give it the whole SM's threads
   const int threads = smem > 96 * 1024 ? 1024 : (smem > 48 * 1024 ? 512 : 256);
-  if (fast_math) scan_select_kernel<true><<<a.R_max, threads, smem, st>>>(a);
-  else scan_select_kernel<false><<<a.R_max, threads, smem, st>>>(a);
+  if (fast_math) launch_pdl(scan_select_kernel<true>, dim3(a.R_max), dim3(threads), smem, st, a);
+  else launch_pdl(scan_select_kernel<false>, dim3(a.R_max), dim3(threads), smem, st, a);
 }
 
 }  // namespace tw

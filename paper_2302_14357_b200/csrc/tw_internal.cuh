@@ -13,6 +13,39 @@ constexpr int kMaxSeg = TW_MAX_SEGMENT;
 constexpr int kMaxLayers = 4;
 
 // ---------------------------------------------------------------------------------------------
+// Programmatic dependent launch.  The kernels of a decode step run back to back on one stream, each
+// reading what the previous one wrote.  Launched with launch_pdl, a kernel may be scheduled while its
+// predecessor is still running (once every CTA of the predecessor has called pdl_trigger or exited), so
+// its set-up (barriers, tensor memory, tensor-map prefetch) overlaps the predecessor's tail.  The rules
+// every kernel launched this way follows: (1) every thread calls pdl_wait before it reads or writes
+// global memory that another kernel of the stream writes or reads, and every CTA calls it on every path
+// (a kernel that finished without waiting would release ITS successor too early); (2) nothing before
+// pdl_wait has a side effect outside the CTA.  pdl_wait returns at once in a kernel launched normally.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// Host-side switch of the calling thread: while false, launch_pdl launches normally.  Two decoders that share
+// the GPU on two streams keep it off: an early-scheduled CTA that only waits would hold an SM the other
+// stream's kernels could use.
+inline thread_local bool g_pdl_on = true;
+struct PdlScope {
+  bool saved;
+  explicit PdlScope(bool on) : saved(g_pdl_on) { g_pdl_on = on; }
+  ~PdlScope() { g_pdl_on = saved; }
+};
+
+template <typename... P, typename... A>
+inline cudaError_t launch_pdl(void (*kern)(P...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, A&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = g_pdl_on ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<P>(args)...);
+}
+
+// ---------------------------------------------------------------------------------------------
 // numerics helpers (accurate libm versions: the fp32 mode must track an fp64 reference to ~1e-6)
 __device__ __forceinline__ float logaddexp_f(float a, float b) {
   if (a == -INFINITY) return b;
