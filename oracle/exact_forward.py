@@ -58,3 +58,38 @@ def brute_force_log_prob(model: rm.RnntModel, enc: np.ndarray, y: Sequence[int])
         return total
 
     return float(np.log(walk(0, 0, 1.0)))
+
+
+def forward_log_prob_monotonic(model: rm.RnntModel, enc: np.ndarray, y: Sequence[int]) -> float:
+    """Monotonic lattice (every output consumes a frame):
+    alpha(t+1, u) = alpha(t, u) J(t, u, blank) + alpha(t, u-1) J(t, u-1, y_u);  p(y|x) = alpha(T, U)."""
+    lj = _lattice_log_probs(model, enc, y)
+    T, U = lj.shape[0], len(y)
+    blank = model.blank
+    alpha = np.full((T + 1, U + 1), -np.inf)
+    alpha[0, 0] = 0.0
+    for t in range(T):
+        for u in range(U + 1):
+            stay = alpha[t, u] + lj[t, u, blank]
+            emit = alpha[t, u - 1] + lj[t, u - 1, y[u - 1]] if u > 0 else -np.inf
+            alpha[t + 1, u] = np.logaddexp(stay, emit)
+    return float(alpha[T, U])
+
+
+def brute_force_log_prob_monotonic(model: rm.RnntModel, enc: np.ndarray, y: Sequence[int]) -> float:
+    """Sum over every way to place the U tokens on distinct frames, in order; all other frames emit blank."""
+    lj = _lattice_log_probs(model, enc, y)
+    J = np.exp(lj)
+    T, U = J.shape[0], len(y)
+    blank = model.blank
+
+    def walk(t: int, u: int, p: float) -> float:
+        if t == T:
+            return p if u == U else 0.0
+        total = walk(t + 1, u, p * J[t, u, blank])
+        if u < U:
+            total += walk(t + 1, u + 1, p * J[t, u, y[u]])
+        return total
+
+    total = walk(0, 0, 1.0)
+    return float(np.log(total)) if total > 0.0 else -np.inf

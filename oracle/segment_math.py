@@ -61,3 +61,35 @@ def blank_expansion(lBl: np.ndarray, ld_old: np.ndarray) -> np.ndarray:
     H, S = ld_old.shape
     terms = np.stack([ld_old[:, t1 - 1] + lBl[:, t1, S + 1] for t1 in range(1, S + 1)], axis=0)
     return logsumexp(terms, axis=0)
+
+
+# ---- monotonic variant (Sec. 2 and Sec. 5 name it as an easy adjustment; the equations below are this
+# code's own derivation, pinned by brute force in the tests) --------------------------------------
+# In a monotonic RNN-T every output, blank or token, consumes one frame.  A hypothesis that emits
+# token k at frame t2 therefore continues at frame t2 + 1, and one that emits at the segment's last
+# frame has left the segment.  Frame distributions get one more entry, index S'+1: "past the segment".
+
+
+def nonblank_expansion_t_monotonic(logJ: np.ndarray, lBl: np.ndarray, ld_old: np.ndarray, blank: int = 0) -> np.ndarray:
+    """Monotonic Eq. 4-5.  ld_old [H, S'+1] -> log d [H, V, S'+1] with
+    d[h, k, t2 + 1] = sum_{t1=1}^{S'} d_old[h, t1] * Bl(h, t1, t2) * J(t2, h, k)   for t2 = 1..S',
+    d[h, k, 1] = 0.  Mass already past the segment (d_old[h, S'+1]) cannot emit here."""
+    H, S, V = logJ.shape
+    assert ld_old.shape == (H, S + 1)
+    ld = np.full((H, V, S + 1), NEG_INF)
+    for t2 in range(1, S + 1):
+        terms = np.full((S, H, V), NEG_INF)
+        for t1 in range(1, S + 1):
+            terms[t1 - 1] = (ld_old[:, t1 - 1] + lBl[:, t1, t2])[:, None] + logJ[:, t2 - 1, :]
+        ld[:, :, t2] = logsumexp(terms, axis=0)          # lands on frame t2 + 1 (array index t2)
+    ld[:, blank, :] = NEG_INF
+    return ld
+
+
+def blank_expansion_monotonic(lBl: np.ndarray, ld_old: np.ndarray) -> np.ndarray:
+    """Monotonic Eq. 7.  delta_phi[h] = sum_{t1=1}^{S'} d_old[h, t1] * Bl(h, t1, S'+1) + d_old[h, S'+1]."""
+    H, S1 = ld_old.shape
+    S = S1 - 1
+    terms = [ld_old[:, t1 - 1] + lBl[:, t1, S + 1] for t1 in range(1, S + 1)]
+    terms.append(ld_old[:, S])
+    return logsumexp(np.stack(terms, axis=0), axis=0)

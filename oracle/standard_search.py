@@ -61,3 +61,35 @@ def standard_beam_search(model: rm.RnntModel, enc: np.ndarray, N: int,
             active = nxt
     ranked = sorted(enumerate(finished.items()), key=lambda e: (-e[1][1][0], e[0]))[:N]
     return [(tok, v[0]) for _, (tok, v) in ranked], calls
+
+
+def monotonic_frame_search(model: rm.RnntModel, enc: np.ndarray, N: int):
+    """Frame-synchronous beam search for a monotonic RNN-T: at every frame each of the N best
+    hypotheses either emits blank or exactly one token, and both consume the frame.  Extensions
+    that spell the same sequence are summed; only the N best token extensions of a frame are formed,
+    and only those that beat the N-th best blank extension (when there are N) are kept."""
+    enc = np.asarray(enc, dtype=np.float64)
+    blank = model.blank
+    st0, o0 = rm.predictor_init(model)
+    beam: Dict[Tuple[int, ...], list] = {(): [0.0, st0, o0]}
+    for t in range(enc.shape[0]):
+        ranked = sorted(enumerate(beam.items()), key=lambda e: (-e[1][1][0], e[0]))[:N]
+        active = [(tok, v[0], v[1], v[2]) for _, (tok, v) in ranked]
+        logJ = rm.joiner_log_probs(model, enc[t:t + 1], np.stack([a[3] for a in active]))[:, 0, :]
+        beam = {}
+        for h, (tok, lp, st, o) in enumerate(active):
+            beam[tok] = [float(lp + logJ[h, blank]), st, o]
+        cands = sorted((-(lp + logJ[h, k]), h, k) for h, (tok, lp, st, o) in enumerate(active)
+                       for k in range(model.V) if k != blank)[:N]
+        stay = sorted((v[0] for v in beam.values()), reverse=True)
+        for neg, h, k in cands:
+            if len(stay) < N or -neg > stay[N - 1]:
+                tok, lp, st, o = active[h]
+                new = tok + (k,)
+                if new in beam:
+                    beam[new][0] = float(np.logaddexp(beam[new][0], -neg))
+                else:
+                    st2, o2 = rm.predictor_step(model, st, k)
+                    beam[new] = [-neg, st2, o2]
+    ranked = sorted(enumerate(beam.items()), key=lambda e: (-e[1][1][0], e[0]))[:N]
+    return [(tok, v[0]) for _, (tok, v) in ranked]

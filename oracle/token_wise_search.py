@@ -12,7 +12,14 @@ Readings of points the paper leaves open (each mirrored by the CUDA path):
     Length(B) < N;
   * the inner loop has a safety cap `max_iters` per segment (the paper relies
     on the threshold alone); hitting it drops the rest of A and is reported;
-  * merged hypotheses keep the predictor state of the entry inserted first.
+  * merged hypotheses keep the predictor state of the entry inserted first;
+  * an expansion of probability zero (log score -inf) is not a hypothesis and is
+    never kept (it only arises in the monotonic variant, from a hypothesis whose
+    whole mass has already left the segment).
+
+`monotonic=True` runs the same loop for a monotonic RNN-T (every output consumes a
+frame): frame distributions carry one more entry for "past the segment" and the
+two monotonic formulas of segment_math replace Eq. 4-5 and Eq. 7.
 
 `DecisionLog` records the score margin of every pruning decision and can
 invert chosen ones, so a test can tell a legitimate near-tie flip of a lower
@@ -116,7 +123,8 @@ def choose_n_best_expansions(ldnb: np.ndarray, n: int, blank: int, log=None) -> 
 def token_wise_beam_search(model: rm.RnntModel, enc: np.ndarray, N: int, S: int,
                            max_iters: Optional[int] = None,
                            max_len: Optional[int] = None,
-                           log: Optional[DecisionLog] = None):
+                           log: Optional[DecisionLog] = None,
+                           monotonic: bool = False):
     """Algorithm 1.  enc [T, D_enc] -> (list of (tokens, log score) best first, stats).
 
     max_iters: safety cap on inner-loop passes per segment (None = uncapped).
@@ -137,7 +145,7 @@ def token_wise_beam_search(model: rm.RnntModel, enc: np.ndarray, N: int, S: int,
         B = []
         t = t + S
         for hyp in A:
-            ld = np.full(Sp, NEG_INF)
+            ld = np.full(Sp + 1 if monotonic else Sp, NEG_INF)
             ld[0] = hyp.ls                       # all mass on the segment's first frame
             hyp.ld = ld
         it = 0
@@ -153,9 +161,13 @@ def token_wise_beam_search(model: rm.RnntModel, enc: np.ndarray, N: int, S: int,
 
             ld_old = np.stack([hyp.ld for hyp in A])              # [H, S']
             lBl = sm.blank_product(logJ, blank)                   # Eq. 3
-            ld_new = sm.nonblank_expansion_t(logJ, lBl, ld_old, blank)  # Eq. 4-5
+            if monotonic:
+                ld_new = sm.nonblank_expansion_t_monotonic(logJ, lBl, ld_old, blank)
+                ldphi = sm.blank_expansion_monotonic(lBl, ld_old)
+            else:
+                ld_new = sm.nonblank_expansion_t(logJ, lBl, ld_old, blank)  # Eq. 4-5
+                ldphi = sm.blank_expansion(lBl, ld_old)           # Eq. 7
             ldnb = sm.nonblank_expansion(ld_new)                  # Eq. 6
-            ldphi = sm.blank_expansion(lBl, ld_old)               # Eq. 7
 
             for h, hyp in enumerate(A):
                 add_and_merge(B, Hypothesis(hyp.tok, float(ldphi[h]), hyp.state, hyp.o, None))
@@ -165,6 +177,8 @@ def token_wise_beam_search(model: rm.RnntModel, enc: np.ndarray, N: int, S: int,
             threshold = choose_nth_score(B, N) if len(B) >= N else None
             for (h, k) in choose_n_best_expansions(ldnb, N, blank, log):
                 score = float(ldnb[h, k])
+                if score == NEG_INF:
+                    continue
                 if max_len is not None and len(A_prev[h].tok) + 1 > max_len:
                     continue
                 if len(B) < N:

@@ -394,3 +394,69 @@ def test_iteration_cap_is_reported():
     cfg, model, enc = tiny_case(V=6, T=6, pred="stateless", seed=4, blank_bias=-3.0)
     _, st = tws.token_wise_beam_search(model, enc, N=2, S=3, max_iters=1)
     assert st.limit_hit and max(st.iters_per_segment) == 1
+
+
+# ---- monotonic variant: every output consumes a frame ------------------------------------------------
+
+@pytest.mark.parametrize("S", [1, 2, 3, 7])
+def test_monotonic_mass_conservation_and_shift(S):
+    """Monotonic segment formulas: mass is conserved (including what has already left the segment), a new
+    hypothesis sits one frame after its emission, and delta_nb equals the standard one on the same input."""
+    rng = np.random.default_rng(40 + S)
+    H, V = 4, 7
+    logJ = _random_logJ(rng, H, S, V)
+    ld_old = rng.standard_normal((H, S + 1)) * 3 - 5
+    ld_old[0, 1:] = -np.inf                       # a hypothesis at segment start
+    ld_old[1, :S] = -np.inf                       # a hypothesis that has left the segment entirely
+    lBl = sm.blank_product(logJ)
+    ld = sm.nonblank_expansion_t_monotonic(logJ, lBl, ld_old)
+    dphi = sm.blank_expansion_monotonic(lBl, ld_old)
+    total = np.logaddexp(dphi, sm.logsumexp(sm.nonblank_expansion(ld)[:, 1:], axis=1))
+    np.testing.assert_allclose(total, sm.logsumexp(ld_old, axis=1), rtol=0, atol=1e-12)
+    assert np.all(np.isneginf(ld[:, :, 0]))       # nothing can sit on the first frame after an emission
+    std = sm.nonblank_expansion_t(logJ, lBl, ld_old[:, :S])
+    np.testing.assert_allclose(ld[:, 1:, 1:], std[:, 1:, :], atol=1e-13)
+    assert dphi[1] == pytest.approx(ld_old[1, S], abs=1e-13) and np.all(np.isneginf(ld[1]))
+    np.testing.assert_allclose(np.exp(dphi), np.exp(sm.blank_expansion(lBl, ld_old[:, :S])) + np.exp(ld_old[:, S]), rtol=1e-12)
+
+
+@pytest.mark.parametrize("pred", ["stateless", "lstm"])
+@pytest.mark.parametrize("T,S", [(4, 1), (4, 2), (4, 3), (4, 4), (6, 4), (5, 2), (3, 50)])
+def test_monotonic_unpruned_search_is_exact(pred, T, S):
+    """Un-pruned, the monotonic search gives every sequence of at most T tokens the sum over all placements
+    of its tokens on distinct frames: forward recursion and brute force agree, for every segment size."""
+    V, U = 4, 3
+    cfg, model, enc = tiny_case(V=V, T=T, pred=pred, seed=T * 10 + S + 500)
+    seqs = [y for y in _all_sequences(V, U) if len(y) <= T]
+    nbest, stats = tws.token_wise_beam_search(model, enc, N=10 * len(seqs) + 10, S=S, max_len=U, monotonic=True)
+    got = dict(nbest)
+    assert set(seqs) <= set(got)
+    for y in seqs:
+        fwd = ef.forward_log_prob_monotonic(model, enc, y)
+        assert got[y] == pytest.approx(fwd, abs=1e-11)
+        assert ef.brute_force_log_prob_monotonic(model, enc, y) == pytest.approx(fwd, abs=1e-11)
+    # a monotonic model spreads all its mass over sequences of at most T tokens
+    if U >= T:
+        assert sum(math.exp(s) for s in got.values()) == pytest.approx(1.0, abs=1e-10)
+    # it is a different lattice from the standard one: the same sequence gets a different probability
+    assert abs(got[(1, 1)] - ef.forward_log_prob(model, enc, (1, 1))) > 1e-6
+
+
+@pytest.mark.parametrize("pred,N", [("stateless", 1), ("stateless", 3), ("lstm", 2), ("lstm", 4)])
+def test_monotonic_segment_size_one_is_the_frame_synchronous_search(pred, N):
+    cfg, model, enc = tiny_case(V=6, T=9, pred=pred, seed=21 + N, blank_bias=1.0)
+    ref = ss.monotonic_frame_search(model, enc, N)
+    got, stats = tws.token_wise_beam_search(model, enc, N=N, S=1, monotonic=True)
+    assert [t for t, _ in got] == [t for t, _ in ref]
+    np.testing.assert_allclose([s for _, s in got], [s for _, s in ref], atol=1e-12)
+    assert all(len(t) <= 9 for t, _ in got)
+
+
+@pytest.mark.parametrize("S", [2, 3, 5, 8])
+def test_monotonic_pruned_scores_never_exceed_exact_probability(S):
+    cfg, model, enc = tiny_case(V=6, T=10, pred="lstm", seed=5, blank_bias=1.5)
+    nbest, stats = tws.token_wise_beam_search(model, enc, N=3, S=S, max_iters=4 * S + 16, monotonic=True)
+    assert len(nbest) == 3 and not stats.limit_hit
+    for y, s in nbest:
+        assert s <= ef.forward_log_prob_monotonic(model, enc, y) + 1e-10
+    assert max(stats.iters_per_segment) <= S + 1     # at most one token per frame, then everything has left
