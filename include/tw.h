@@ -278,6 +278,14 @@ int tw_set_graph(tw_handle* h, int on);
  * tw_set_lanes(h, 0) decodes the batch in one piece.  Default: on.  Off while profiling is on. */
 int tw_set_lanes(tw_handle* h, int on);
 
+/* Monotonic RNN-T variant (Sec. 2 and Sec. 5 name it as an adjustment of Algorithm 1; the paper prints no
+ * equations for it).  Every output, blank or token, consumes one frame, so at most one token is emitted
+ * per frame.  In Eq. 4-5 a token emitted at frame t2 leaves its hypothesis at frame t2 + 1, and a
+ * hypothesis that emits at the segment's last frame has left the segment: its mass is added to Eq. 7's
+ * delta_phi.  Eq. 3 and Eq. 6 are unchanged.  on != 0 selects the variant for later tw_decode and
+ * tw_stream_open calls on this handle; TW_ERR_STATE while a streaming session is open.  Default: off. */
+int tw_set_monotonic(tw_handle* h, int on);
+
 /* Per-stage device timing of tw_decode with CUDA events on the decode stream (adds two event records
  * per stage per step); off by default. */
 int tw_set_profiling(tw_handle* h, int on);

@@ -79,7 +79,8 @@ def _ordered_top(scores: Sequence[float], n: int, log: Optional[DecisionLog], ki
     order = sorted(range(len(scores)), key=lambda i: (-scores[i], i))
     if len(order) > n:
         if log is not None and n >= 1:
-            gap = scores[order[n - 1]] - scores[order[n]]
+            # a cut below which everything has probability zero is no decision: its margin is infinite
+            gap = scores[order[n - 1]] - scores[order[n]] if scores[order[n]] > NEG_INF else np.inf
             if log.decide(kind, gap):
                 order[n - 1], order[n] = order[n], order[n - 1]
         order = order[:n]

@@ -12,7 +12,7 @@ TW_OK, TW_ERR_ARG, TW_ERR_ALLOC, TW_ERR_CUDA, TW_ERR_LIMIT, TW_ERR_STATE, TW_ERR
 
 EXPORTED_SYMBOLS = [
     "tw_init", "tw_destroy", "tw_decode", "tw_decode_host", "tw_max_tokens", "tw_project_encoder",
-    "tw_joiner_segment", "tw_expand", "tw_joiner_expand", "tw_predictor_step", "tw_get_stats", "tw_set_profiling", "tw_set_fused", "tw_set_graph", "tw_set_lanes",
+    "tw_joiner_segment", "tw_expand", "tw_joiner_expand", "tw_predictor_step", "tw_get_stats", "tw_set_profiling", "tw_set_fused", "tw_set_graph", "tw_set_lanes", "tw_set_monotonic",
     "tw_stream_open", "tw_stream_push", "tw_stream_nbest", "tw_stream_close",
     "tw_joiner_expand_noalloc",
     "tw_last_cuda_error", "tw_strerror",
@@ -73,6 +73,7 @@ def load_library() -> C.CDLL:
     lib.tw_set_fused.argtypes = [vp, C.c_int]
     lib.tw_set_graph.argtypes = [vp, C.c_int]
     lib.tw_set_lanes.argtypes = [vp, C.c_int]
+    lib.tw_set_monotonic.argtypes = [vp, C.c_int]
     lib.tw_stream_open.argtypes = [vp, i32, vp]
     lib.tw_stream_push.argtypes = [vp, vp, vp, i32, vp]
     lib.tw_stream_nbest.argtypes = [vp, vp, vp, vp, vp, vp]
@@ -287,6 +288,10 @@ class TwDecoder:
 
     def set_graph(self, on: bool):
         self._check(self.lib.tw_set_graph(self.h, int(bool(on))), "tw_set_graph")
+
+    def set_monotonic(self, on: bool):
+        """tw_set_monotonic: the monotonic RNN-T variant (every output consumes a frame) for later decodes."""
+        self._check(self.lib.tw_set_monotonic(self.h, int(bool(on))), "tw_set_monotonic")
 
     def set_lanes(self, on: bool):
         self._check(self.lib.tw_set_lanes(self.h, int(bool(on))), "tw_set_lanes")

@@ -39,6 +39,7 @@ __device__ void turn_over(const HypState& hs, int b) {
         const int slot = hs.B_slot[(long long)b * hs.capB + e];
         hs.A_slot[b * kMaxBeam + i] = slot;
         hs.A_ls[b * kMaxBeam + i] = hs.B_ls[(long long)b * hs.capB + e];
+        hs.A_done[b * kMaxBeam + i] = -INFINITY;
         hs.carry[b * kMaxBeam + i] = slot;
       } else {
         hs.carry[b * kMaxBeam + i] = -1;
@@ -90,7 +91,7 @@ constexpr int kStepThreads = 512;   // 16 warps: one per hypothesis of list A
 __global__ void __launch_bounds__(kStepThreads) hyp_step_kernel(HypState hs) {
   __shared__ int s_nB, s_hasthr, s_nkeep;
   __shared__ int s_found[kMaxBeam], s_touched[kMaxBeam], s_carry[kMaxBeam];
-  __shared__ double s_Als[kMaxBeam];
+  __shared__ double s_Als[kMaxBeam], s_Adone[kMaxBeam];
   __shared__ int s_Aslot[kMaxBeam];
   __shared__ double s_thr;
   __shared__ int s_ck[kMaxBeam * kMaxBeam];
@@ -113,7 +114,10 @@ __global__ void __launch_bounds__(kStepThreads) hyp_step_kernel(HypState hs) {
   const long long bS = (long long)b * hs.capSlot;
 
   if (tid < kMaxBeam) {
-    if (tid < H) { s_Als[tid] = hs.A_ls[b * kMaxBeam + tid]; s_Aslot[tid] = hs.A_slot[b * kMaxBeam + tid]; }
+    if (tid < H) {
+      s_Als[tid] = hs.A_ls[b * kMaxBeam + tid]; s_Aslot[tid] = hs.A_slot[b * kMaxBeam + tid];
+      s_Adone[tid] = hs.mono ? hs.A_done[b * kMaxBeam + tid] : -INFINITY;
+    }
     s_carry[tid] = hs.carry[b * kMaxBeam + tid];
   }
   if (tid == 0) { hs.calls[b] += 1; hs.joins[b] += slen; }
@@ -150,7 +154,8 @@ __global__ void __launch_bounds__(kStepThreads) hyp_step_kernel(HypState hs) {
   if (tid < H) {
     const int h = tid;
     const int slot = s_Aslot[h];
-    const double val = s_Als[h] + (hs.ldphi_d ? hs.ldphi_d[r0 + h] : (double)hs.ldphi[r0 + h]);
+    double val = s_Als[h] + (hs.ldphi_d ? hs.ldphi_d[r0 + h] : (double)hs.ldphi[r0 + h]);
+    val = logaddexp_d(val, s_Adone[h]);       // monotonic: plus what had already left the segment (else log 0)
     int e = s_found[h];
     if (e >= 0) {
       hs.B_ls[bB + e] = logaddexp_d(hs.B_ls[bB + e], val);
@@ -271,18 +276,24 @@ __global__ void __launch_bounds__(kStepThreads) hyp_step_kernel(HypState hs) {
       hs.A_ls[b * kMaxBeam + i] = s_keep_ls[i];
     }
     const long long r = r0 + h;
-    for (int t = lane; t < S; t += 32) {
-      double v = -INFINITY;
-      if (t < slen) {
-        const double a = hs.la_d ? hs.la_d[r * S + t] : (double)hs.la[r * S + t];
-        v = s_Als[h] + a;
-        if (hs.logp != nullptr) {      // otherwise log J(t, k) is added by a follow-up kernel
-          double lj = (double)hs.logp[(r * S + t) * V + k];
-          if (hs.lse) lj -= (double)hs.lse[r * S + t];
-          v += lj;
-        }
+    // d_h(k) at frame t of the segment: occupancy times J(t, k)
+    auto d_at = [&](int t) -> double {
+      if (t < 0 || t >= slen) return -INFINITY;
+      const double a = hs.la_d ? hs.la_d[r * S + t] : (double)hs.la[r * S + t];
+      double v = s_Als[h] + a;
+      if (hs.logp != nullptr) {      // otherwise log J(t, k) is added by a follow-up kernel
+        double lj = (double)hs.logp[(r * S + t) * V + k];
+        if (hs.lse) lj -= (double)hs.lse[r * S + t];
+        v += lj;
       }
-      hs.A_ld[((long long)b * kMaxBeam + i) * S + t] = v;
+      return v;
+    };
+    if (!hs.mono) {
+      for (int t = lane; t < S; t += 32) hs.A_ld[((long long)b * kMaxBeam + i) * S + t] = d_at(t);
+    } else {
+      // emitted at frame t: the hypothesis continues at frame t + 1, or has left the segment
+      for (int t = lane; t < S; t += 32) hs.A_ld[((long long)b * kMaxBeam + i) * S + t] = t < slen ? d_at(t - 1) : -INFINITY;
+      if (lane == 0) hs.A_done[b * kMaxBeam + i] = d_at(slen - 1);
     }
   }
   // ---- list A empty: this segment is done ------------------------------------------------------

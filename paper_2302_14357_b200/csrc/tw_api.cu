@@ -238,6 +238,8 @@ int build_workspace(tw_handle* h) {
   TW_TRY(dev_alloc(h, &hs.A_slot, nb * kMaxBeam));
   TW_TRY(dev_alloc(h, &hs.A_ls, nb * kMaxBeam));
   TW_TRY(dev_alloc(h, &hs.A_ld, nb * kMaxBeam * S));
+  TW_TRY(dev_alloc(h, &hs.A_done, nb * kMaxBeam));
+  hs.mono = 0;
   TW_TRY(dev_alloc(h, &hs.B_slot, nB));
   TW_TRY(dev_alloc(h, &hs.B_ls, nB));
   TW_TRY(dev_alloc(h, &hs.B_hash, nB));
@@ -473,6 +475,19 @@ int tw_set_fused(tw_handle* h, int on) {
   if (!h) return TW_ERR_ARG;
   if (on && !h->bf.fused_ok) return TW_ERR_STATE;
   h->bf.fused_on = on != 0;
+  return TW_OK;
+}
+
+int tw_set_monotonic(tw_handle* h, int on) {
+  if (!h) return TW_ERR_ARG;
+  if (h->stream_B > 0) return TW_ERR_STATE;        // not in the middle of a streaming session
+  tw_handle* all[3] = {h, h->lane[0], h->lane[1]};
+  for (tw_handle* x : all) {
+    if (!x) continue;
+    x->hs.mono = x->hs_fused.mono = on ? 1 : 0;
+    // a captured step graph holds the kernels' arguments by value: capture again with the new setting
+    if (x->graph_exec) { cudaGraphExecDestroy(x->graph_exec); x->graph_exec = nullptr; }
+  }
   return TW_OK;
 }
 

@@ -144,6 +144,10 @@ struct HypState {
   int* avail;    // streaming: frames pushed so far (len is the part of them that may be decoded now)
   // list A: [B][kMaxBeam]
   int* A_slot; double* A_ls; double* A_ld;   // A_ld [B][kMaxBeam][S]
+  // Monotonic variant (every output consumes a frame): a token emitted at frame t leaves its hypothesis at
+  // frame t + 1, so A_ld is filled one entry later and A_done [B][kMaxBeam] holds the mass that has left the
+  // segment (emitted at its last frame), which joins delta_phi.  mono == 0: A_done is unused.
+  double* A_done; int mono;
   // list B of Algorithm 1 (hypotheses finished for this segment): [B][capB]
   int* B_slot; double* B_ls; unsigned long long* B_hash; int* B_len;
   int* B_top;    // [B][kMaxBeam] indices into list B of its best entries, best first

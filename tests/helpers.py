@@ -52,20 +52,21 @@ def _same_nbest(ref, got, tol, tau):
     return True
 
 
-def check_against_oracle(model, enc, N, S, max_iters, got, tol=SCORE_TOL, tau=TIE_TAU, max_flips=6):
+def check_against_oracle(model, enc, N, S, max_iters, got, tol=SCORE_TOL, tau=TIE_TAU, max_flips=6, monotonic=False):
     """Runs Algorithm 1 in the oracle and compares with `got`.  Returns (ok, how, stats) where how is
     'exact' or 'near-tie' (the oracle reproduces `got` after inverting one or two pruning decisions
     whose score gap is below tau)."""
     import itertools
     from oracle import token_wise_search as tws
     log = tws.DecisionLog()
-    ref, stats = tws.token_wise_beam_search(model, enc, N, S, max_iters=max_iters, log=log)
+    ref, stats = tws.token_wise_beam_search(model, enc, N, S, max_iters=max_iters, log=log, monotonic=monotonic)
     if _same_nbest(ref, got, tol, tau):
         return True, "exact", stats
     close = log.below(tau)[:max_flips]
     for n in (1, 2):
         for flips in itertools.combinations(close, n):
-            ref2, _ = tws.token_wise_beam_search(model, enc, N, S, max_iters=max_iters, log=tws.DecisionLog(flips))
+            ref2, _ = tws.token_wise_beam_search(model, enc, N, S, max_iters=max_iters, log=tws.DecisionLog(flips),
+                                                 monotonic=monotonic)
             if _same_nbest(ref2, got, tol, tau):
                 return True, "near-tie", stats
     return False, "mismatch: oracle %r vs %r (min margin %.3g)" % (ref[:2], got[:2], log.min_margin()), stats
