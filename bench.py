@@ -40,6 +40,7 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-lanes", action="store_true", help="decode the batch in one piece instead of two concurrent halves")
     ap.add_argument("--no-fused", action="store_true", help="bf16 mode: staged joiner kernels instead of the fused one")
+    ap.add_argument("--monotonic", action="store_true", help="the monotonic RNN-T variant (every output consumes a frame)")
     ap.add_argument("--cpu-frames", type=int, default=0, help="frames of the CPU-baseline sample (0: auto)")
     return ap.parse_args()
 
@@ -76,7 +77,7 @@ def measured_peaks():
 
 # ------------------------------------------------------------------------------------------------
 # CPU baseline: the oracle as it stands, on a bounded sample of the same workload
-def oracle_sample(cfg, S, frames, utt=0):
+def oracle_sample(cfg, S, frames, utt=0, monotonic=False):
     from oracle import rnnt_model as rm
     from oracle import token_wise_search as tws
     try:
@@ -90,7 +91,7 @@ def oracle_sample(cfg, S, frames, utt=0):
                       activation=cfg.joiner_act)
     n = int(min(frames, lens[utt]))
     t0 = time.perf_counter()
-    _, st = tws.token_wise_beam_search(om, enc[utt, :n], cfg.N, S, max_iters=4 * S + 16)
+    _, st = tws.token_wise_beam_search(om, enc[utt, :n], cfg.N, S, max_iters=4 * S + 16, monotonic=monotonic)
     dt = time.perf_counter() - t0
     return {"value": n / dt, "unit": UNIT, "cores": int(cores), "kind": "oracle",
             "sample": "utterance %d of workload %s, first %d frames, N=%d S=%d, fp64 numpy; %.1f s"
@@ -111,10 +112,10 @@ def run_reference(args, cfg, S):
         return
     frames = args.cpu_frames or max(12, auto_cpu_frames(cfg) // 4)
     for _ in range(args.warmup):
-        oracle_sample(cfg, S, max(4, frames // 4))
+        oracle_sample(cfg, S, max(4, frames // 4), monotonic=args.monotonic)
     times, vals, last = [], [], None
     for k in range(args.steps):
-        last, dt = oracle_sample(cfg, S, frames, utt=0)
+        last, dt = oracle_sample(cfg, S, frames, utt=0, monotonic=args.monotonic)
         times.append(dt)
         vals.append(last["value"])
     value = frames * len(times) / sum(times) if times else 0.0
@@ -123,7 +124,8 @@ def run_reference(args, cfg, S):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": 1e3 * sum(times) / max(len(times), 1), "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": cfg.name, "N": cfg.N, "S": S, "sample_frames_per_step": frames},
+            "config": {"workload": cfg.name, "N": cfg.N, "S": S, "sample_frames_per_step": frames,
+                       "variant": "monotonic" if args.monotonic else "standard"},
             "cpu_baseline": base,
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
@@ -204,6 +206,8 @@ def run_ours(args, cfg, S):
         dec.set_fused(False)
     if args.no_lanes:
         dec.set_lanes(False)
+    if args.monotonic:
+        dec.set_monotonic(True)
     enc = torch.from_numpy(enc_np).cuda()
     lens = torch.from_numpy(len_np).cuda()
     frames = int(len_np.sum())
@@ -281,7 +285,7 @@ def run_ours(args, cfg, S):
         "ms_per_step": ms / args.steps, "ms_per_step_with_stage_events": ms_profiled / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": mode_name, "data": "synthetic",
         "config": {"workload": cfg.name, "B_per_gpu": B, "T": cfg.T, "N": cfg.N, "S": S, "J": cfg.J, "V": cfg.V,
-                   "mode": mode_name, "l2": ("inputs larger than L2 (encoder batch %.0f MB)" % (enc_np.nbytes / 1e6)) if flush is None
+                   "mode": mode_name, "variant": "monotonic" if args.monotonic else "standard", "l2": ("inputs larger than L2 (encoder batch %.0f MB)" % (enc_np.nbytes / 1e6)) if flush is None
                          else "L2 flushed by a 256 MB write before every timed step (encoder batch %.0f MB)" % (enc_np.nbytes / 1e6),
                    "parallelism": "independent utterance batches per GPU, no collective"},
         "calls_per_frame": st["calls"] / max(st["frames"], 1), "joins_per_frame": st["joins"] / max(st["frames"], 1),
@@ -300,7 +304,7 @@ def run_ours(args, cfg, S):
         "clocks": clocks,
     }
     if not args.no_cpu_baseline and world == 1:
-        line["cpu_baseline"], _ = oracle_sample(cfg, S, args.cpu_frames or auto_cpu_frames(cfg))
+        line["cpu_baseline"], _ = oracle_sample(cfg, S, args.cpu_frames or auto_cpu_frames(cfg), monotonic=args.monotonic)
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
