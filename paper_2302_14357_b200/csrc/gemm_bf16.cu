@@ -223,7 +223,7 @@ constexpr size_t kWideSmem = (size_t)kWideStages * (kWideABytes + kWideBBytes) +
 
 __global__ void __launch_bounds__(kThreadsWide, 1)
 gemm_lstm_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB64,
-                      const __grid_constant__ CUtensorMap tmB32, GemmBf16Params p, int n_split) {
+                      const __grid_constant__ CUtensorMap tmB32, GemmBf16Params p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* sA = smem;
@@ -233,11 +233,6 @@ gemm_lstm_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
   uint64_t* acc_full = empty + kWideStages;
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(acc_full + 1);
 
-  const int mt = blockIdx.x / n_split, ns = blockIdx.x - mt * n_split;
-  const int m0 = mt * BM;
-  const int units = p.N >> 5, ubase = units / n_split, urem = units - ubase * n_split;
-  const int u0 = ns * ubase + (ns < urem ? ns : urem), nu = ubase + (ns < urem ? 1 : 0);
-  const int n0 = u0 * 32, w = nu * 32;                   // this CTA's columns [n0, n0 + w), w <= kWideMaxBN
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_kb = (p.K + BK - 1) / BK;
 
@@ -258,8 +253,20 @@ gemm_lstm_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
   // the set-up above touched only this CTA: it may overlap the tail of the kernel that produces A and M
   pdl_wait();
   pdl_trigger();
+  // The split follows the row count of THIS launch: fewer row tiles than the grid was sized for give
+  // every row tile more CTAs, i.e. narrower and faster tiles (never wider than the host's bound).
   const int M = p.M_dev ? *p.M_dev : p.M;
-  const bool active = m0 < M && nu > 0;                  // an idle CTA skips the roles and only frees its TMEM
+  const int m_tiles = M > 0 ? (M + BM - 1) / BM : 1;
+  const int units = p.N >> 5;
+  int n_split = (int)gridDim.x / m_tiles;
+  n_split = n_split < 1 ? 1 : (n_split > units ? units : n_split);
+  const int mt = blockIdx.x / n_split, ns = blockIdx.x - mt * n_split;
+  const int m0 = mt * BM;
+  const int ubase = units / n_split, urem = units - ubase * n_split;
+  const int u0 = ns * ubase + (ns < urem ? ns : urem), nu = ubase + (ns < urem ? 1 : 0);
+  const int n0 = u0 * 32, w = nu * 32;                   // this CTA's columns [n0, n0 + w), w <= kWideMaxBN
+  if (w > kWideMaxBN && threadIdx.x == 0) atomicExch(p.err, 1);    // the host sizes the grid so that this cannot happen
+  const bool active = m0 < M && mt < m_tiles && w <= kWideMaxBN;   // an idle CTA skips the roles and only frees its TMEM
 
   if (!active) {
   } else if (warp == 0) {
@@ -432,7 +439,7 @@ bool launch_gemm_lstm_wide(const CUtensorMap& tmA, const CUtensorMap& tmB64, con
   if (n_split < 1) return false;
   const int units = p.N >> 5;
   if (((units + n_split - 1) / n_split) * 32 > kWideMaxBN) return false;
-  launch_pdl(gemm_lstm_wide_kernel, dim3(mt * n_split), dim3(kThreadsWide), kWideSmem, st, tmA, tmB64, tmB32, p, n_split);
+  launch_pdl(gemm_lstm_wide_kernel, dim3(mt * n_split), dim3(kThreadsWide), kWideSmem, st, tmA, tmB64, tmB32, p);
   return true;
 }
 
