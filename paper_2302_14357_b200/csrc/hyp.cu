@@ -303,41 +303,47 @@ __global__ void __launch_bounds__(kStepThreads) hyp_step_kernel(HypState hs) {
 // One CTA: packs the live hypotheses of all utterances into joiner rows and the new hypotheses
 // into the predictor's work list.
 __global__ void __launch_bounds__(1024) compact_kernel(HypState hs, int B, int T) {
-  __shared__ int s_a[1024], s_n[1024];
+  __shared__ int s_wa[32], s_wn[32];       // per-warp totals of the two scans
+  __shared__ int s_cnt[1024], s_off[1024]; // batches of up to 1024 utterances: nA | n_new << 8, row_off | new_off << 16 kept on chip
   __shared__ int s_base_a, s_base_n, s_frames;
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   pdl_wait();
   pdl_trigger();
   if (tid == 0) { s_base_a = 0; s_base_n = 0; s_frames = 0; }
   __syncthreads();
-  // exclusive scans of the list sizes -> row_off, new_off
+  // exclusive scans of the list sizes -> row_off, new_off (shuffle scan per warp, then over the warp totals)
   for (int b0 = 0; b0 < B; b0 += 1024) {
     const int b = b0 + tid;
     const int a = b < B ? hs.nA[b] : 0;
     const int nn = b < B ? hs.n_new[b] : 0;
-    s_a[tid] = a; s_n[tid] = nn;
-    __syncthreads();
-    for (int o = 1; o < 1024; o <<= 1) {
-      int va = 0, vn = 0;
-      if (tid >= o) { va = s_a[tid - o]; vn = s_n[tid - o]; }
-      __syncthreads();
-      s_a[tid] += va; s_n[tid] += vn;
-      __syncthreads();
+    const int fr = (b < B && a > 0) ? a * hs.slen[b] : 0;
+    int ia = a, in = nn;                   // inclusive scans inside the warp
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int va = __shfl_up_sync(0xffffffffu, ia, o), vn = __shfl_up_sync(0xffffffffu, in, o);
+      if (lane >= o) { ia += va; in += vn; }
     }
+    if (lane == 31) { s_wa[warp] = ia; s_wn[warp] = in; }
+    if (fr > 0) atomicAdd(&s_frames, fr);
+    __syncthreads();
+    int pa = 0, pn = 0;                    // totals of the warps before this one
+    for (int w = 0; w < warp; ++w) { pa += s_wa[w]; pn += s_wn[w]; }
     if (b < B) {
-      hs.row_off[b] = s_base_a + s_a[tid] - a;
-      hs.new_off[b] = s_base_n + s_n[tid] - nn;
-      if (a > 0) atomicAdd(&s_frames, a * hs.slen[b]);
+      hs.row_off[b] = s_base_a + pa + ia - a;
+      hs.new_off[b] = s_base_n + pn + in - nn;
+      if (B <= 1024) { s_cnt[tid] = a | (nn << 8); s_off[tid] = (pa + ia - a) | ((pn + in - nn) << 16); }
     }
     __syncthreads();
-    if (tid == 1023) { s_base_a += s_a[1023]; s_base_n += s_n[1023]; }
+    if (tid == 1023) { s_base_a += pa + ia; s_base_n += pn + in; }
     __syncthreads();
   }
   // fill: one thread per (utterance, list position)
   for (int idx = tid; idx < B * kMaxBeam; idx += 1024) {
     const int b = idx / kMaxBeam, h = idx % kMaxBeam;
-    if (h < hs.nA[b]) {
-      const int r = hs.row_off[b] + h;
+    const bool chip = B <= 1024;           // offsets fit 16 bits: at most 1024 * kMaxBeam rows
+    const int nA_b = chip ? (s_cnt[b] & 255) : hs.nA[b], nnew_b = chip ? (s_cnt[b] >> 8) : hs.n_new[b];
+    if (h < nA_b) {
+      const int r = (chip ? (s_off[b] & 0xffff) : hs.row_off[b]) + h;
       const int slot = hs.A_slot[b * kMaxBeam + h];
       const long long gs = (long long)b * hs.capSlot + slot;
       hs.row_b[r] = b;
@@ -355,8 +361,8 @@ __global__ void __launch_bounds__(1024) compact_kernel(HypState hs, int B, int T
         hs.row_ld[(long long)r * hs.S + t] = (d == -INFINITY) ? -INFINITY : (float)(d - ls);
       }
     }
-    if (h < hs.n_new[b]) {
-      const int o = hs.new_off[b] + h;
+    if (h < nnew_b) {
+      const int o = (chip ? (s_off[b] >> 16) : hs.new_off[b]) + h;
       hs.pw_new[o] = hs.new_slot[b * kMaxBeam + h];
       hs.pw_par[o] = hs.new_par[b * kMaxBeam + h];
       hs.pw_tok[o] = hs.new_tok[b * kMaxBeam + h];
