@@ -26,36 +26,37 @@ __device__ __forceinline__ unsigned long long hash_push(unsigned long long h, in
 // Starts the next segment of utterance b: A = ChooseNBest(B), B = [], t += S, d = (s, 0, ..., 0).
 // Precondition: list A is empty and frames remain.  Called by the whole CTA.
 __device__ void turn_over(const HypState& hs, int b) {
-  __shared__ int s_n;
+  __shared__ double s_ls[kMaxBeam];
+  __syncthreads();
+  const int n = hs.nTop[b];                  // read by every thread before thread 0 clears it below
+  if (threadIdx.x < kMaxBeam) {              // one thread per carried hypothesis
+    const int i = threadIdx.x;
+    if (i < n) {
+      const int e = hs.B_top[b * kMaxBeam + i];
+      const int slot = hs.B_slot[(long long)b * hs.capB + e];
+      const double ls = hs.B_ls[(long long)b * hs.capB + e];
+      hs.A_slot[b * kMaxBeam + i] = slot;
+      hs.A_ls[b * kMaxBeam + i] = ls;
+      hs.A_done[b * kMaxBeam + i] = -INFINITY;
+      hs.carry[b * kMaxBeam + i] = slot;
+      s_ls[i] = ls;
+    } else {
+      hs.carry[b * kMaxBeam + i] = -1;
+    }
+  }
   __syncthreads();
   if (threadIdx.x == 0) {
-    const int n = hs.nTop[b];
     const int t0 = hs.t0[b] + hs.slen[b];
     hs.t0[b] = t0;
     hs.slen[b] = min(hs.S, hs.len[b] - t0);
-    for (int i = 0; i < kMaxBeam; ++i) {
-      if (i < n) {
-        const int e = hs.B_top[b * kMaxBeam + i];
-        const int slot = hs.B_slot[(long long)b * hs.capB + e];
-        hs.A_slot[b * kMaxBeam + i] = slot;
-        hs.A_ls[b * kMaxBeam + i] = hs.B_ls[(long long)b * hs.capB + e];
-        hs.A_done[b * kMaxBeam + i] = -INFINITY;
-        hs.carry[b * kMaxBeam + i] = slot;
-      } else {
-        hs.carry[b * kMaxBeam + i] = -1;
-      }
-    }
     hs.nA[b] = n;
     hs.nB[b] = 0;
     hs.nTop[b] = 0;
     hs.iters[b] = 0;
-    s_n = n;
   }
-  __syncthreads();
-  const int n = s_n;
   for (int i = threadIdx.x; i < n * hs.S; i += blockDim.x) {
     const int a = i / hs.S, t = i - a * hs.S;
-    hs.A_ld[((long long)b * kMaxBeam + a) * hs.S + t] = (t == 0) ? hs.A_ls[b * kMaxBeam + a] : -INFINITY;
+    hs.A_ld[((long long)b * kMaxBeam + a) * hs.S + t] = (t == 0) ? s_ls[a] : -INFINITY;
   }
 }
 
@@ -92,7 +93,7 @@ __global__ void __launch_bounds__(kStepThreads) hyp_step_kernel(HypState hs) {
   __shared__ int s_nB, s_hasthr, s_nkeep;
   __shared__ int s_found[kMaxBeam], s_touched[kMaxBeam], s_carry[kMaxBeam];
   __shared__ double s_Als[kMaxBeam], s_Adone[kMaxBeam];
-  __shared__ int s_Aslot[kMaxBeam];
+  __shared__ int s_Aslot[kMaxBeam], s_Alen[kMaxBeam];
   __shared__ double s_thr;
   __shared__ int s_ck[kMaxBeam * kMaxBeam];
   __shared__ double s_abs[kMaxBeam * kMaxBeam];
@@ -147,7 +148,7 @@ __global__ void __launch_bounds__(kStepThreads) hyp_step_kernel(HypState hs) {
         if (!__any_sync(0xffffffffu, diff)) found = c;
       }
     }
-    if (lane == 0) s_found[warp] = found;
+    if (lane == 0) { s_found[warp] = found; s_Alen[warp] = ln; }
   }
   __syncthreads();
   // ---- AddAndMerge, apply: sum into the matching entry or append (appends keep the order of A)
@@ -236,7 +237,7 @@ __global__ void __launch_bounds__(kStepThreads) hyp_step_kernel(HypState hs) {
       const double sc = s_abs[c];
       if (hasthr && !(sc > thr)) continue;            // Length(B) < N or delta_nb > threshold
       if (capped) { hs.status[b] = TW_ERR_LIMIT; break; }
-      if (hs.slot_len[bS + s_Aslot[h]] + 1 > hs.U_cap) { hs.status[b] = TW_ERR_LIMIT; continue; }
+      if (s_Alen[h] + 1 > hs.U_cap) { hs.status[b] = TW_ERR_LIMIT; continue; }
       // next free slot of the ring: skip slots still held by hypotheses carried into this segment
       bool busy;
       do {
