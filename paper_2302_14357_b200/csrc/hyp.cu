@@ -89,6 +89,13 @@ __global__ void __launch_bounds__(kThreads) hyp_init_kernel(HypState hs, const i
 
 constexpr int kStepThreads = 512;   // 16 warps: one per hypothesis of list A
 
+// Order-preserving integer image of a score: a < b as doubles <=> order_key(a) < order_key(b) as unsigned
+// integers (-0 counts as +0; scores are never NaN).  The ranking loops compare these instead of doubles.
+__device__ __forceinline__ unsigned long long order_key(double x) {
+  const unsigned long long u = (unsigned long long)__double_as_longlong(x + 0.0);
+  return (u >> 63) ? ~u : (u | 0x8000000000000000ull);
+}
+
 __global__ void __launch_bounds__(kStepThreads) hyp_step_kernel(HypState hs) {
   __shared__ int s_nB, s_hasthr, s_nkeep;
   __shared__ int s_found[kMaxBeam], s_touched[kMaxBeam], s_carry[kMaxBeam];
@@ -97,6 +104,9 @@ __global__ void __launch_bounds__(kStepThreads) hyp_step_kernel(HypState hs) {
   __shared__ double s_thr;
   __shared__ int s_ck[kMaxBeam * kMaxBeam];
   __shared__ double s_abs[kMaxBeam * kMaxBeam];
+  __shared__ unsigned long long s_key[kMaxBeam * kMaxBeam];
+  __shared__ unsigned long long s_nkey[32];
+  __shared__ int s_nidx[32];
   __shared__ int s_sel[kMaxBeam];
   __shared__ int s_keep_h[kMaxBeam], s_keep_k[kMaxBeam], s_keep_slot[kMaxBeam];
   __shared__ double s_keep_ls[kMaxBeam];
@@ -189,11 +199,15 @@ __global__ void __launch_bounds__(kStepThreads) hyp_step_kernel(HypState hs) {
       if (!dup) idx = cand;
     }
     const double score = idx >= 0 ? hs.B_ls[bB + idx] : -INFINITY;
+    const unsigned long long key = order_key(score);
+    s_nkey[lane] = key; s_nidx[lane] = idx;
+    __syncwarp();
     int rank = 0;
-    for (int j = 0; j < 32; ++j) {
-      const double sj = __shfl_sync(0xffffffffu, score, j);
-      const int ij = __shfl_sync(0xffffffffu, idx, j);
-      if (ij >= 0 && (sj > score || (sj == score && ij < idx))) ++rank;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {          // all lanes read the same word: broadcasts, independent of each other
+      const unsigned long long kj = s_nkey[j];
+      const int ij = s_nidx[j];
+      rank += (ij >= 0 && (kj > key || (kj == key && ij < idx))) ? 1 : 0;
     }
     const int count = __popc(__ballot_sync(0xffffffffu, idx >= 0));
     __syncwarp();
@@ -208,15 +222,20 @@ __global__ void __launch_bounds__(kStepThreads) hyp_step_kernel(HypState hs) {
     const bool valid = h < H && j < hs.cand_n[r0 + h];
     s_abs[tid] = valid ? s_Als[h] + (double)hs.cand_v[(long long)(r0 + h) * kMaxBeam + j] : -INFINITY;
     s_ck[tid] = valid ? hs.cand_k[(long long)(r0 + h) * kMaxBeam + j] : -1;
+    s_key[tid] = order_key(s_abs[tid]);
   }
   if (tid < kMaxBeam) s_sel[tid] = -1;
   __syncthreads();
   if (tid < kMaxBeam * kMaxBeam && s_ck[tid] >= 0) {
-    const double mine = s_abs[tid];
+    const unsigned long long mine = s_key[tid];
     int rank = 0;
-    for (int o = 0; o < kMaxBeam * kMaxBeam; ++o) {
-      const double so = s_abs[o];
-      if (s_ck[o] >= 0 && (so > mine || (so == mine && o < tid))) ++rank;
+    for (int hh = 0; hh < H; ++hh) {         // rows past H hold no candidate
+#pragma unroll
+      for (int j = 0; j < kMaxBeam; ++j) {
+        const int o = hh * kMaxBeam + j;
+        const unsigned long long so = s_key[o];
+        rank += (s_ck[o] >= 0 && (so > mine || (so == mine && o < tid))) ? 1 : 0;
+      }
     }
     if (rank < N) s_sel[rank] = tid;
   }
