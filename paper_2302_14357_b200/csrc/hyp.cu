@@ -107,6 +107,8 @@ __global__ void __launch_bounds__(kStepThreads) hyp_step_kernel(HypState hs) {
   __shared__ unsigned long long s_key[kMaxBeam * kMaxBeam];
   __shared__ unsigned long long s_nkey[32];
   __shared__ int s_nidx[32];
+  __shared__ int s_cursor, s_iters, s_nT0, s_Btop[kMaxBeam];     // per-utterance state fetched up front
+  __shared__ double s_Btopls[kMaxBeam], s_tval[kMaxBeam];         // scores of B's old best / of the entries touched now
   __shared__ int s_sel[kMaxBeam];
   __shared__ int s_keep_h[kMaxBeam], s_keep_k[kMaxBeam], s_keep_slot[kMaxBeam];
   __shared__ double s_keep_ls[kMaxBeam];
@@ -132,6 +134,17 @@ __global__ void __launch_bounds__(kStepThreads) hyp_step_kernel(HypState hs) {
     s_carry[tid] = hs.carry[b * kMaxBeam + tid];
   }
   if (tid == 0) { hs.calls[b] += 1; hs.joins[b] += slen; }
+  if (warp == 15) {
+    // ring cursor, pass counter and the best-N set of list B as the previous pass left it: fetched now, by a
+    // warp that has nothing to do in the search, so that the later phases find them in shared memory
+    const int nT = hs.nTop[b];
+    if (lane == 0) { s_cursor = hs.cursor[b]; s_iters = hs.iters[b]; s_nT0 = nT; }
+    if (lane < kMaxBeam) {
+      const int bt = hs.B_top[b * kMaxBeam + lane];
+      s_Btop[lane] = bt;
+      if (lane < nT) s_Btopls[lane] = hs.B_ls[bB + bt];       // before this pass's merges; touched entries are patched below
+    }
+  }
   __syncthreads();
 
   // ---- AddAndMerge, search: warp h looks for the tokens of A_h among the entries already in B.
@@ -169,7 +182,8 @@ __global__ void __launch_bounds__(kStepThreads) hyp_step_kernel(HypState hs) {
     val = logaddexp_d(val, s_Adone[h]);       // monotonic: plus what had already left the segment (else log 0)
     int e = s_found[h];
     if (e >= 0) {
-      hs.B_ls[bB + e] = logaddexp_d(hs.B_ls[bB + e], val);
+      val = logaddexp_d(hs.B_ls[bB + e], val);
+      hs.B_ls[bB + e] = val;
     } else {
       e = nB0;                              // capB = N * I_max bounds this by construction
       for (int q = 0; q < h; ++q) e += (s_found[q] < 0);
@@ -177,6 +191,7 @@ __global__ void __launch_bounds__(kStepThreads) hyp_step_kernel(HypState hs) {
       hs.B_hash[bB + e] = hs.slot_hash[bS + slot]; hs.B_len[bB + e] = hs.slot_len[bS + slot];
     }
     s_touched[h] = e;
+    s_tval[h] = val;
   }
   if (tid == 0) {
     int nB = nB0;
@@ -188,17 +203,19 @@ __global__ void __launch_bounds__(kStepThreads) hyp_step_kernel(HypState hs) {
 
   // ---- ChooseNthScore: the best N of B are among the previous best N and the entries touched now
   if (warp == 0) {
-    const int nT = hs.nTop[b];
+    const int nT = s_nT0;
     int idx = -1;
+    double score = -INFINITY;
     if (lane < nT) {
-      idx = hs.B_top[b * kMaxBeam + lane];
+      idx = s_Btop[lane];
+      score = s_Btopls[lane];
+      for (int q = 0; q < H; ++q) if (s_touched[q] == idx) score = s_tval[q];   // merged into in this pass
     } else if (lane - nT < H) {
       const int cand = s_touched[lane - nT];
       bool dup = false;
-      for (int i = 0; i < nT; ++i) dup |= (hs.B_top[b * kMaxBeam + i] == cand);
-      if (!dup) idx = cand;
+      for (int i = 0; i < nT; ++i) dup |= (s_Btop[i] == cand);
+      if (!dup) { idx = cand; score = s_tval[lane - nT]; }
     }
-    const double score = idx >= 0 ? hs.B_ls[bB + idx] : -INFINITY;
     const unsigned long long key = order_key(score);
     s_nkey[lane] = key; s_nidx[lane] = idx;
     __syncwarp();
@@ -229,12 +246,14 @@ __global__ void __launch_bounds__(kStepThreads) hyp_step_kernel(HypState hs) {
   if (tid < kMaxBeam * kMaxBeam && s_ck[tid] >= 0) {
     const unsigned long long mine = s_key[tid];
     int rank = 0;
-    for (int hh = 0; hh < H; ++hh) {         // rows past H hold no candidate
+    // rows past H hold no candidate; an empty entry has the key of log 0, which ranks below every candidate
+    // (candidates are finite), so it needs no validity test
+    for (int hh = 0; hh < H; ++hh) {
 #pragma unroll
       for (int j = 0; j < kMaxBeam; ++j) {
         const int o = hh * kMaxBeam + j;
         const unsigned long long so = s_key[o];
-        rank += (s_ck[o] >= 0 && (so > mine || (so == mine && o < tid))) ? 1 : 0;
+        rank += (so > mine || (so == mine && o < tid)) ? 1 : 0;
       }
     }
     if (rank < N) s_sel[rank] = tid;
@@ -243,34 +262,37 @@ __global__ void __launch_bounds__(kStepThreads) hyp_step_kernel(HypState hs) {
   const bool hasthr = s_hasthr != 0;
   const double thr = hasthr ? s_thr : -INFINITY;
 
-  // ---- filter against the threshold, allocate slots ------------------------------------------
-  if (tid == 0) {
-    int nk = 0;
-    int cur = hs.cursor[b];
-    const bool capped = hs.iters[b] + 1 >= hs.I_max;
-    hs.iters[b] += 1;
-    for (int i = 0; i < N; ++i) {
-      const int c = s_sel[i];
-      if (c < 0) break;
-      const int h = c / kMaxBeam;
-      const double sc = s_abs[c];
-      if (hasthr && !(sc > thr)) continue;            // Length(B) < N or delta_nb > threshold
-      if (capped) { hs.status[b] = TW_ERR_LIMIT; break; }
-      if (s_Alen[h] + 1 > hs.U_cap) { hs.status[b] = TW_ERR_LIMIT; continue; }
-      // next free slot of the ring: skip slots still held by hypotheses carried into this segment
-      bool busy;
-      do {
+  // ---- filter against the threshold, allocate slots: lane i of warp 0 takes the i-th best expansion
+  if (warp == 0) {
+    const int c = lane < N ? s_sel[lane] : -1;
+    const int h = c >= 0 ? c / kMaxBeam : 0;
+    const double sc = c >= 0 ? s_abs[c] : -INFINITY;
+    const bool pass = c >= 0 && (!hasthr || sc > thr);      // Length(B) < N or delta_nb > threshold
+    const bool capped = s_iters + 1 >= hs.I_max;
+    const bool fits = s_Alen[h] + 1 <= hs.U_cap;
+    const bool keep = pass && !capped && fits;
+    const unsigned passm = __ballot_sync(0xffffffffu, pass), keepm = __ballot_sync(0xffffffffu, keep);
+    const int nk = __popc(keepm), m = __popc(keepm & ((1u << lane) - 1u));
+    if (keep) {
+      // the (m + 1)-th free slot of the ring after the cursor: slots still held by hypotheses carried into
+      // this segment are skipped
+      int cur = s_cursor, need = m + 1;
+      while (need > 0) {
         cur = (cur + 1 == hs.capSlot) ? 0 : cur + 1;
-        busy = false;
+        bool busy = false;
 #pragma unroll
         for (int q = 0; q < kMaxBeam; ++q) busy |= (s_carry[q] == cur);
-      } while (busy);
-      s_keep_h[nk] = h; s_keep_k[nk] = s_ck[c]; s_keep_ls[nk] = sc; s_keep_slot[nk] = cur;
-      ++nk;
+        if (!busy) --need;
+      }
+      s_keep_h[m] = h; s_keep_k[m] = s_ck[c]; s_keep_ls[m] = sc; s_keep_slot[m] = cur;
+      if (m == nk - 1) hs.cursor[b] = cur;
     }
-    hs.cursor[b] = cur;
-    s_nkeep = nk;
-    hs.nA[b] = nk; hs.n_new[b] = nk;
+    if (lane == 0) {
+      hs.iters[b] = s_iters + 1;
+      if (passm != 0 && (capped || (passm & ~keepm) != 0)) hs.status[b] = TW_ERR_LIMIT;   // pass cap or token capacity
+      s_nkeep = nk;
+      hs.nA[b] = nk; hs.n_new[b] = nk;
+    }
   }
   __syncthreads();
   const int nk = s_nkeep;
