@@ -77,7 +77,7 @@ __device__ __forceinline__ float window_sum(float x, int S) {
 #pragma unroll
   for (int size = 1; size <= 32; size <<= 1) {
     if (size > SS) break;
-    if (SS & size) { total += __shfl_down_sync(0xffffffffu, cur, off); off += size; }
+    if (SS & size) { total += (off == 0) ? cur : __shfl_down_sync(0xffffffffu, cur, off); off += size; }   // the first piece is the lane's own
     if (2 * size <= SS) cur += __shfl_down_sync(0xffffffffu, cur, size);
   }
   return total;
