@@ -327,6 +327,10 @@ gemm_lstm_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         prefetch_l2(cin + ((n0 + c * 32) >> 2));
       }
     }
+    // 256-bit accesses when every row segment this kernel touches starts on a 32-byte boundary
+    const bool wide_ok = (p.lstm.Hd & 7) == 0 &&
+                         ((reinterpret_cast<uintptr_t>(p.lstm.hc_in) | reinterpret_cast<uintptr_t>(p.lstm.hc_out) |
+                           reinterpret_cast<uintptr_t>(p.addend) | (uintptr_t)(p.ld_add * 4)) & 31) == 0;
     bool ok = mbar_wait(acc_full, 0, p.err);
     ok = __all_sync(0xffffffffu, ok);
     if (ok) {
@@ -344,15 +348,29 @@ gemm_lstm_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             v[j] += b4.x; v[j + 1] += b4.y; v[j + 2] += b4.z; v[j + 3] += b4.w;
           }
         }
-        if (arow) {
+        float cp[8];
+        if (wide_ok) {
+          if (arow) {
 #pragma unroll
-          for (int j = 0; j < 32; j += 4) {
-            const float4 a4 = __ldg(reinterpret_cast<const float4*>(arow + nb + j));
-            v[j] += a4.x; v[j + 1] += a4.y; v[j + 2] += a4.z; v[j + 3] += a4.w;
+            for (int j = 0; j < 32; j += 8) {
+              float a8[8];
+              ld_global_v8(arow + nb + j, a8);
+#pragma unroll
+              for (int u = 0; u < 8; ++u) v[j + u] += a8[u];
+            }
           }
+          ld_global_v8(cin + j0, cp);
+        } else {
+          if (arow) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 4) {
+              const float4 a4 = __ldg(reinterpret_cast<const float4*>(arow + nb + j));
+              v[j] += a4.x; v[j + 1] += a4.y; v[j + 2] += a4.z; v[j + 3] += a4.w;
+            }
+          }
+          const float4 c0 = *reinterpret_cast<const float4*>(cin + j0), c1 = *reinterpret_cast<const float4*>(cin + j0 + 4);
+          cp[0] = c0.x; cp[1] = c0.y; cp[2] = c0.z; cp[3] = c0.w; cp[4] = c1.x; cp[5] = c1.y; cp[6] = c1.z; cp[7] = c1.w;
         }
-        const float4 c0 = *reinterpret_cast<const float4*>(cin + j0), c1 = *reinterpret_cast<const float4*>(cin + j0 + 4);
-        const float cp[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
         float hn[8], cn[8];
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
@@ -361,10 +379,15 @@ gemm_lstm_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
           hn[u] = sigmoid_fast(v[4 * u + 3]) * tanh_fast_g(cc);
         }
         float* cout = hout + p.lstm.Hd;
-        *reinterpret_cast<float4*>(hout + j0) = make_float4(hn[0], hn[1], hn[2], hn[3]);
-        *reinterpret_cast<float4*>(hout + j0 + 4) = make_float4(hn[4], hn[5], hn[6], hn[7]);
-        *reinterpret_cast<float4*>(cout + j0) = make_float4(cn[0], cn[1], cn[2], cn[3]);
-        *reinterpret_cast<float4*>(cout + j0 + 4) = make_float4(cn[4], cn[5], cn[6], cn[7]);
+        if (wide_ok) {
+          st_global_v8(hout + j0, hn);
+          st_global_v8(cout + j0, cn);
+        } else {
+          *reinterpret_cast<float4*>(hout + j0) = make_float4(hn[0], hn[1], hn[2], hn[3]);
+          *reinterpret_cast<float4*>(hout + j0 + 4) = make_float4(hn[4], hn[5], hn[6], hn[7]);
+          *reinterpret_cast<float4*>(cout + j0) = make_float4(cn[0], cn[1], cn[2], cn[3]);
+          *reinterpret_cast<float4*>(cout + j0 + 4) = make_float4(cn[4], cn[5], cn[6], cn[7]);
+        }
         __nv_bfloat162 b0 = __floats2bfloat162_rn(hn[0], hn[1]), b1 = __floats2bfloat162_rn(hn[2], hn[3]);
         __nv_bfloat162 b2 = __floats2bfloat162_rn(hn[4], hn[5]), b3 = __floats2bfloat162_rn(hn[6], hn[7]);
         uint4 pk;
