@@ -157,22 +157,45 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
               for (int j = 0; j < 32; ++j) v[j] += p.bias[nb + j];
             }
             if (arow) {
+              if ((reinterpret_cast<uintptr_t>(arow + nb) & 31) == 0) {
 #pragma unroll
-              for (int j = 0; j < 32; ++j) v[j] += arow[nb + j];
+                for (int j = 0; j < 32; j += 8) {
+                  float a8[8];
+                  ld_global_v8(arow + nb + j, a8);
+#pragma unroll
+                  for (int u = 0; u < 8; ++u) v[j + u] += a8[u];
+                }
+              } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] += arow[nb + j];
+              }
             }
             const int j0 = nb >> 2;
-            float hn[8], cn[8];
+            const bool w256 = (p.lstm.Hd & 7) == 0 &&
+                              ((reinterpret_cast<uintptr_t>(p.lstm.hc_in) | reinterpret_cast<uintptr_t>(p.lstm.hc_out)) & 31) == 0;
+            float cp[8], hn[8], cn[8];
+            if (w256) {
+              ld_global_v8(cin + j0, cp);
+            } else {
+#pragma unroll
+              for (int u = 0; u < 8; ++u) cp[u] = cin[j0 + u];
+            }
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
-              const float c = sigmoid_fast(v[4 * u + 1]) * cin[j0 + u] + sigmoid_fast(v[4 * u]) * tanh_fast_g(v[4 * u + 2]);
+              const float c = sigmoid_fast(v[4 * u + 1]) * cp[u] + sigmoid_fast(v[4 * u]) * tanh_fast_g(v[4 * u + 2]);
               cn[u] = c;
               hn[u] = sigmoid_fast(v[4 * u + 3]) * tanh_fast_g(c);
             }
             float* cout = hout + p.lstm.Hd;
-            *reinterpret_cast<float4*>(hout + j0) = make_float4(hn[0], hn[1], hn[2], hn[3]);
-            *reinterpret_cast<float4*>(hout + j0 + 4) = make_float4(hn[4], hn[5], hn[6], hn[7]);
-            *reinterpret_cast<float4*>(cout + j0) = make_float4(cn[0], cn[1], cn[2], cn[3]);
-            *reinterpret_cast<float4*>(cout + j0 + 4) = make_float4(cn[4], cn[5], cn[6], cn[7]);
+            if (w256) {
+              st_global_v8(hout + j0, hn);
+              st_global_v8(cout + j0, cn);
+            } else {
+              *reinterpret_cast<float4*>(hout + j0) = make_float4(hn[0], hn[1], hn[2], hn[3]);
+              *reinterpret_cast<float4*>(hout + j0 + 4) = make_float4(hn[4], hn[5], hn[6], hn[7]);
+              *reinterpret_cast<float4*>(cout + j0) = make_float4(cn[0], cn[1], cn[2], cn[3]);
+              *reinterpret_cast<float4*>(cout + j0 + 4) = make_float4(cn[4], cn[5], cn[6], cn[7]);
+            }
             __nv_bfloat162 b0 = __floats2bfloat162_rn(hn[0], hn[1]), b1 = __floats2bfloat162_rn(hn[2], hn[3]);
             __nv_bfloat162 b2 = __floats2bfloat162_rn(hn[4], hn[5]), b3 = __floats2bfloat162_rn(hn[6], hn[7]);
             uint4 pk;
@@ -187,12 +210,27 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
               for (int j = 0; j < 32; ++j) v[j] += p.bias[nb + j];
             }
             if (arow) {
+              if ((reinterpret_cast<uintptr_t>(arow + nb) & 31) == 0) {
 #pragma unroll
-              for (int j = 0; j < 32; ++j) v[j] += arow[nb + j];
+                for (int j = 0; j < 32; j += 8) {
+                  float a8[8];
+                  ld_global_v8(arow + nb + j, a8);
+#pragma unroll
+                  for (int u = 0; u < 8; ++u) v[j + u] += a8[u];
+                }
+              } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] += arow[nb + j];
+              }
             }
+            if ((reinterpret_cast<uintptr_t>(crow + nb) & 31) == 0) {   // a thread writes its own row: 32-byte sectors
 #pragma unroll
-            for (int j = 0; j < 32; j += 4)
-              *reinterpret_cast<float4*>(crow + nb + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+              for (int j = 0; j < 32; j += 8) st_global_v8(crow + nb + j, &v[j]);
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; j += 4)
+                *reinterpret_cast<float4*>(crow + nb + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+            }
           } else {
             for (int j = 0; j < 32; ++j)
               if (nb + j < p.N) crow[nb + j] = v[j] + (p.bias ? p.bias[nb + j] : 0.f) + (arow ? arow[nb + j] : 0.f);
