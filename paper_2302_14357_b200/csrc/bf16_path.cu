@@ -38,8 +38,21 @@ __global__ void gather_parents_bf16_kernel(GatherParents g, const int* n_dev, in
   if (r >= n) return;
   const float* src = g.hc + (long long)(g.idx ? g.idx[r] : r) * g.stride + (long long)l * 2 * g.Hd;
   __nv_bfloat16* d = g.dst[l] + (long long)r * g.ld[l] + g.off[l];
-  for (int k = threadIdx.x * 2; k < g.Hd; k += blockDim.x * 2)
-    *reinterpret_cast<__nv_bfloat162*>(d + k) = __floats2bfloat162_rn(src[k], src[k + 1]);
+  // Hd is a multiple of 8 in bf16 mode (the operands' K must be): 8 floats in, one 16-byte store out per thread
+  if (((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(d)) & 15) == 0 && (g.Hd & 7) == 0) {
+    for (int k = threadIdx.x * 8; k < g.Hd; k += blockDim.x * 8) {
+      const float4 a = *reinterpret_cast<const float4*>(src + k), b = *reinterpret_cast<const float4*>(src + k + 4);
+      __nv_bfloat162 p0 = __floats2bfloat162_rn(a.x, a.y), p1 = __floats2bfloat162_rn(a.z, a.w);
+      __nv_bfloat162 p2 = __floats2bfloat162_rn(b.x, b.y), p3 = __floats2bfloat162_rn(b.z, b.w);
+      uint4 pk;
+      pk.x = *reinterpret_cast<uint32_t*>(&p0); pk.y = *reinterpret_cast<uint32_t*>(&p1);
+      pk.z = *reinterpret_cast<uint32_t*>(&p2); pk.w = *reinterpret_cast<uint32_t*>(&p3);
+      *reinterpret_cast<uint4*>(d + k) = pk;
+    }
+  } else {
+    for (int k = threadIdx.x * 2; k < g.Hd; k += blockDim.x * 2)
+      *reinterpret_cast<__nv_bfloat162*>(d + k) = __floats2bfloat162_rn(src[k], src[k + 1]);
+  }
 }
 
 __global__ void permute_cols_f32_kernel(const float* __restrict__ src, const int* __restrict__ perm, long long rows,
