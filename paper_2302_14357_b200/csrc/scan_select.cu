@@ -55,7 +55,8 @@ __global__ void __launch_bounds__(kMaxT) scan_select_kernel(ScanSelectArgs a) {
   const int S = a.S, V = a.V, blank = a.blank;
   const int sl = a.dnb_in ? 1 : (a.row_slen ? a.row_slen[r] : S);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int kT = blockDim.x, nwarps = kT >> 5, ngroups = kT >> 4;
+  const int kT = blockDim.x, nwarps = kT >> 5;
+  const int gshift = kT >= 256 ? 4 : 3, ngroups = kT >> gshift;   // groups of 16 threads (8 in a 128-thread CTA): at least 16 groups
   const float* z = a.z + (long long)r * S * V;
 
   float tmax = -INFINITY;
@@ -155,9 +156,8 @@ __global__ void __launch_bounds__(kMaxT) scan_select_kernel(ScanSelectArgs a) {
 
   // ---- a lower bound of the row's N-th best value: the N-th largest of 16 group maxima (each is a
   // distinct element of the row), so everything at or above it is a small superset of the answer
-#pragma unroll
-  for (int o = 8; o > 0; o >>= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
-  if ((tid & 15) == 0) s_gmax[tid >> 4] = tmax;
+  for (int o = (1 << gshift) >> 1; o > 0; o >>= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
+  if ((tid & ((1 << gshift) - 1)) == 0) s_gmax[tid >> gshift] = tmax;
   __syncthreads();
   if (warp == 0) {
     for (int g = lane; g < ngroups; g += 32) {
@@ -250,7 +250,8 @@ void launch_scan_select(const ScanSelectArgs& a, bool fast_math, cudaStream_t st
   if (a.R_max <= 0) return;
   const size_t smem = a.dnb_in ? scan_select_smem_bytes(1, a.V) : scan_select_smem_bytes(a.S, a.V);
   // a row that takes most of an SM's shared memory runs alone there: give it the whole SM's threads
-  const int threads = smem > 96 * 1024 ? 1024 : (smem > 48 * 1024 ? 512 : 256);
+  // selection from a short row (delta_nb given): 128-thread CTAs, so that a whole batch of rows is resident at once
+  const int threads = smem > 96 * 1024 ? 1024 : (smem > 48 * 1024 ? 512 : ((a.dnb_in && smem <= 16 * 1024) ? 128 : 256));
   if (fast_math) launch_pdl(scan_select_kernel<true>, dim3(a.R_max), dim3(threads), smem, st, a);
   else launch_pdl(scan_select_kernel<false>, dim3(a.R_max), dim3(threads), smem, st, a);
 }
