@@ -397,10 +397,12 @@ __global__ void __launch_bounds__(1024) compact_kernel(HypState hs, int B, int T
       } else {
         hs.row_p[r] = (int)gs;
       }
-      const double ls = hs.A_ls[b * kMaxBeam + h];
-      for (int t = 0; t < hs.S; ++t) {
-        const double d = hs.A_ld[((long long)b * kMaxBeam + h) * hs.S + t];
-        hs.row_ld[(long long)r * hs.S + t] = (d == -INFINITY) ? -INFINITY : (float)(d - ls);
+      if (!hs.defer_rows) {
+        const double ls = hs.A_ls[b * kMaxBeam + h];
+        for (int t = 0; t < hs.S; ++t) {
+          const double d = hs.A_ld[((long long)b * kMaxBeam + h) * hs.S + t];
+          hs.row_ld[(long long)r * hs.S + t] = (d == -INFINITY) ? -INFINITY : (float)(d - ls);
+        }
       }
     }
     if (h < nnew_b) {
@@ -411,7 +413,7 @@ __global__ void __launch_bounds__(1024) compact_kernel(HypState hs, int B, int T
     }
   }
   __syncthreads();
-  for (int b = tid; b < B; b += 1024) hs.n_new[b] = 0;
+  if (!hs.defer_rows) for (int b = tid; b < B; b += 1024) hs.n_new[b] = 0;
   if (tid == 0) {
     const int R = s_base_a;
     hs.scalars[kScR] = R;

@@ -216,8 +216,16 @@ int build_bf16(tw_handle* h) {
       h->bf.fused_on = fused_joiner_specialised(h->S);
     }
   }
+  h->hs.defer_rows = 0;
   h->hs_fused = h->hs;
   h->hs_fused.logp = nullptr; h->hs_fused.lse = nullptr; h->hs_fused.ldphi_d = nullptr; h->hs_fused.la_d = nullptr;
+  if (h->mode == TW_MODE_BF16 && h->bf.fused_ok) {
+    h->aux_ok = cudaStreamCreateWithFlags(&h->aux_stream, cudaStreamNonBlocking) == cudaSuccess &&
+                cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) == cudaSuccess &&
+                cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming) == cudaSuccess;
+    if (!h->aux_ok) cudaGetLastError();
+    h->hs_fused.defer_rows = h->aux_ok ? 1 : 0;
+  }
   TW_CUDA(h, cudaGetLastError());
   return TW_OK;
 }
@@ -370,8 +378,12 @@ void enqueue_scan(tw_handle* h, const JoinerRows& rows, const float* ld_old, flo
 
 // Fused path: joiner, softmax, Eq. 3-7 and per-row candidates with the logits kept in tensor memory
 int enqueue_joiner_fused(tw_handle* h, const JoinerRows& rows, const float* ld_old, float* ldphi, float* ldnb,
-                         float* la, const CandOut& cand, cudaStream_t st, int* launches, StageMarkFn mark_fn) {
-  launch_joiner_A_tiled(rows, h->bf.A_tiled.ptr, st);
+                         float* la, const CandOut& cand, cudaStream_t st, int* launches, StageMarkFn mark_fn,
+                         bool plain_first) {
+  {
+    PdlScope first(plain_first ? false : g_pdl_on);
+    launch_joiner_A_tiled(rows, h->bf.A_tiled.ptr, st);
+  }
   if (mark_fn) mark_fn(h, 3, st);       // operand preparation is booked with the elementwise stages
   if (ldnb == nullptr) ldnb = h->hs.ldnb;
   FusedJoinerParams fp{};
@@ -462,6 +474,9 @@ int tw_destroy(tw_handle* h) {
   if (h->graph_exec) cudaGraphExecDestroy(h->graph_exec);
   if (h->ev_order) cudaEventDestroy(h->ev_order);
   if (h->ev_poll) cudaEventDestroy(h->ev_poll);
+  if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+  if (h->ev_join) cudaEventDestroy(h->ev_join);
+  if (h->aux_stream) cudaStreamDestroy(h->aux_stream);
   if (h->own_stream) cudaStreamDestroy(h->own_stream);
   if (h->host_flag) cudaFreeHost(h->host_flag);
   delete h;

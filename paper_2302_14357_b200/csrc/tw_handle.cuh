@@ -60,6 +60,12 @@ struct tw_handle {
   cudaGraphExec_t graph_exec = nullptr;
   int graph_B = -1, graph_T = -1, graph_fused = -1, graph_launches = 0;
   cudaEvent_t ev_poll = nullptr;
+  // side branch of a decode step: the kernel that completes the new hypotheses' frame distributions and
+  // writes the rows' row_ld runs on aux_stream beside the next pass's predictor kernels (fork after the
+  // compaction kernel, join before the joiner's operand kernel)
+  cudaStream_t aux_stream = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+  bool aux_ok = false, aux_pending = false;
 
   // state of the decode in flight (decode_begin .. decode_end)
   struct Run {
@@ -91,7 +97,8 @@ void enqueue_joiner_logits(tw_handle* h, const JoinerRows& rows, float* logp, cu
 // mark_fn (optional) is called with stage 3 after the operand kernel and stage 2 after the fused kernel
 typedef void (*StageMarkFn)(tw_handle*, int, cudaStream_t);
 int enqueue_joiner_fused(tw_handle* h, const JoinerRows& rows, const float* ld_old, float* ldphi, float* ldnb,
-                         float* la, const CandOut& cand, cudaStream_t st, int* launches, StageMarkFn mark_fn = nullptr);
+                         float* la, const CandOut& cand, cudaStream_t st, int* launches, StageMarkFn mark_fn = nullptr,
+                         bool plain_first = false);   // plain_first: the operand kernel is launched with plain stream ordering
 void enqueue_scan(tw_handle* h, const JoinerRows& rows, const float* ld_old, float* logp, float* ldphi,
                   float* ldnb, float* la, double* ldphi_d, double* la_d, const CandOut& cand, cudaStream_t st,
                   int* launches);
