@@ -100,7 +100,7 @@ void launch_joiner_A_tiled(const JoinerRows& rows, __nv_bfloat16* A, cudaStream_
 int launch_fused_joiner(const CUtensorMap& tmA, const CUtensorMap& tmB256, const FusedJoinerParams& p,
                         int max_clusters, cudaStream_t st);
 // adds log J(t, parent row, token) to A_ld of the hypotheses created in this step
-void launch_survivor_ld(const HypState& hs, int B, const __nv_bfloat16* A, const __nv_bfloat16* W, const float* bias,
+void launch_survivor_ld(const HypState& hs, int B, int T, const __nv_bfloat16* A, const __nv_bfloat16* W, const float* bias,
                         const float* lse, cudaStream_t st);
 
 }  // namespace tw

@@ -384,7 +384,7 @@ __global__ void __launch_bounds__(1024) compact_kernel(HypState hs, int B, int T
     const int b = idx / kMaxBeam, h = idx % kMaxBeam;
     const bool chip = B <= 1024;           // offsets fit 16 bits: at most 1024 * kMaxBeam rows
     const int nA_b = chip ? (s_cnt[b] & 255) : hs.nA[b], nnew_b = chip ? (s_cnt[b] >> 8) : hs.n_new[b];
-    if (h < nA_b) {
+    if (h < nA_b && !hs.defer_rows) {
       const int r = (chip ? (s_off[b] & 0xffff) : hs.row_off[b]) + h;
       const int slot = hs.A_slot[b * kMaxBeam + h];
       const long long gs = (long long)b * hs.capSlot + slot;
@@ -397,12 +397,10 @@ __global__ void __launch_bounds__(1024) compact_kernel(HypState hs, int B, int T
       } else {
         hs.row_p[r] = (int)gs;
       }
-      if (!hs.defer_rows) {
-        const double ls = hs.A_ls[b * kMaxBeam + h];
-        for (int t = 0; t < hs.S; ++t) {
-          const double d = hs.A_ld[((long long)b * kMaxBeam + h) * hs.S + t];
-          hs.row_ld[(long long)r * hs.S + t] = (d == -INFINITY) ? -INFINITY : (float)(d - ls);
-        }
+      const double ls = hs.A_ls[b * kMaxBeam + h];
+      for (int t = 0; t < hs.S; ++t) {
+        const double d = hs.A_ld[((long long)b * kMaxBeam + h) * hs.S + t];
+        hs.row_ld[(long long)r * hs.S + t] = (d == -INFINITY) ? -INFINITY : (float)(d - ls);
       }
     }
     if (h < nnew_b) {

@@ -148,8 +148,9 @@ struct HypState {
   // frame t + 1, so A_ld is filled one entry later and A_done [B][kMaxBeam] holds the mass that has left the
   // segment (emitted at its last frame), which joins delta_phi.  mono == 0: A_done is unused.
   double* A_done; int mono;
-  // defer_rows != 0: compact_kernel leaves row_ld (and the clearing of n_new) to the kernel that completes the
-  // new hypotheses' frame distributions, which then runs beside the predictor kernels of the next pass
+  // defer_rows != 0: compact_kernel only numbers the rows and builds the predictor's work list; the row tables,
+  // row_ld and the clearing of n_new are left to the kernel that completes the new hypotheses' frame
+  // distributions, which then runs beside the predictor kernels of the next pass
   int defer_rows;
   // list B of Algorithm 1 (hypotheses finished for this segment): [B][capB]
   int* B_slot; double* B_ls; unsigned long long* B_hash; int* B_len;
