@@ -33,10 +33,46 @@ __global__ void gather_concat_bf16_kernel(const float* __restrict__ src1, const 
 __global__ void gather_parents_bf16_kernel(GatherParents g, const int* n_dev, int n_max) {
   pdl_wait();
   pdl_trigger();
-  const int n = n_dev ? *n_dev : n_max;
   const int r = blockIdx.x, l = blockIdx.y;
-  if (r >= n) return;
-  const float* src = g.hc + (long long)(g.idx ? g.idx[r] : r) * g.stride + (long long)l * 2 * g.Hd;
+  int n, parent;
+  if (g.wl.B > 0) {
+    // scan of n_new: each thread sums a contiguous run of utterances, then the runs are scanned
+    __shared__ int s_run[128], s_hit[2], s_total;
+    const int B = g.wl.B, per = (B + blockDim.x - 1) / blockDim.x;
+    const int b0 = threadIdx.x * per, b1 = min(b0 + per, B);
+    int mine = 0;
+    for (int b = b0; b < b1; ++b) mine += g.wl.n_new[b];
+    s_run[threadIdx.x] = mine;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int acc = 0;
+      for (int i = 0; i < (int)blockDim.x; ++i) { const int v = s_run[i]; s_run[i] = acc; acc += v; }
+      s_total = acc;
+    }
+    __syncthreads();
+    n = s_total;
+    if (r == 0 && l == 0 && threadIdx.x == 0) *g.wl.n_out = n;
+    if (r >= n) return;
+    int off = s_run[threadIdx.x];
+    for (int b = b0; b < b1; ++b) {
+      const int nb = g.wl.n_new[b];
+      if (r >= off && r < off + nb) { s_hit[0] = b; s_hit[1] = r - off; }   // exactly one thread, one utterance
+      off += nb;
+    }
+    __syncthreads();
+    const int e = s_hit[0] * kMaxBeam + s_hit[1];
+    parent = g.wl.new_par[e];
+    if (l == 0 && threadIdx.x == 0) {
+      g.wl.pw_new[r] = g.wl.new_slot[e];
+      g.wl.pw_par[r] = parent;
+      g.wl.pw_tok[r] = g.wl.new_tok[e];
+    }
+  } else {
+    n = n_dev ? *n_dev : n_max;
+    if (r >= n) return;
+    parent = g.idx ? g.idx[r] : r;
+  }
+  const float* src = g.hc + (long long)parent * g.stride + (long long)l * 2 * g.Hd;
   __nv_bfloat16* d = g.dst[l] + (long long)r * g.ld[l] + g.off[l];
   // Hd is a multiple of 8 in bf16 mode (the operands' K must be): 8 floats in, one 16-byte store out per thread
   if (((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(d)) & 15) == 0 && (g.Hd & 7) == 0) {

@@ -64,10 +64,20 @@ void launch_gather_concat_bf16(const float* src1, const int* idx1, long long ld1
                                const int* idx2, long long ld2, int K2, const int* n_dev, int n_max,
                                __nv_bfloat16* dst, cudaStream_t st);
 // X[l][r, off_l : off_l + Hd] = bf16(h of layer l in state row (idx ? idx[r] : r)), for every layer at once
+// Optional: the kernel first builds the predictor's work list itself.  Entry r is the i-th new hypothesis of
+// utterance b, where r = (sum of n_new over the utterances before b) + i; every CTA finds its (b, i) by a scan
+// of n_new (B values), the CTAs of layer 0 write entry r of pw_new / pw_par / pw_tok, and CTA (0, 0) writes the
+// list's length to n_out.  B == 0: the list exists already (idx, n_dev).
+struct WorkListBuild {
+  int B;
+  const int* n_new; const int* new_slot; const int* new_par; const int* new_tok;   // [B], [B][kMaxBeam] x 3
+  int* pw_new; int* pw_par; int* pw_tok; int* n_out;
+};
 struct GatherParents {
   const float* hc; const int* idx; long long stride;   // state rows [L][2][Hd]
   int L, Hd;
   __nv_bfloat16* dst[kMaxLayers]; int ld[kMaxLayers]; int off[kMaxLayers];
+  WorkListBuild wl;
 };
 void launch_gather_parents_bf16(const GatherParents& g, const int* n_dev, int n_max, cudaStream_t st);
 // dst[r, c] = src[r, perm[c]]  (fp32, rows x cols)

@@ -67,7 +67,7 @@ void gemm_bf16(tw_handle* h, const Bf16Mat& A, const Bf16Mat& B, const int* M_de
 // output W_p g goes to row (idx_out ? idx_out[i] : i) of Pp_out.  State rows are [L][2][Hd].
 void enqueue_predictor(tw_handle* h, const int* tok, const float* hc_in, const int* idx_in, float* hc_out,
                        const int* idx_out, float* Pp_out, const int* n_dev, int n_max, cudaStream_t st,
-                       int* launches) {
+                       int* launches, const WorkListBuild* wl = nullptr) {
   GemmOperand none{};
   if (h->pred_kind == TW_PRED_STATELESS) {
     GemmOperand a{h->emb, tok, h->emb_dim, h->W_p, h->P, h->P};
@@ -83,6 +83,7 @@ void enqueue_predictor(tw_handle* h, const int* tok, const float* hc_in, const i
     GatherParents g{};
     g.hc = hc_in; g.idx = idx_in; g.stride = stride; g.L = L; g.Hd = Hd;
     for (int l = 0; l < L; ++l) { g.dst[l] = h->bf.X[l].ptr; g.ld[l] = (int)h->bf.X[l].K; g.off[l] = (l == 0) ? 0 : Hd; }
+    if (wl) g.wl = *wl;                       // the gather kernel builds tok / idx_in / idx_out / *n_dev first
     launch_gather_parents_bf16(g, n_dev, n_max, st);
     // gate GEMMs with the LSTM cell in the epilogue; each writes the next GEMM's input half as bf16
     for (int l = 0; l < L; ++l) {
@@ -127,11 +128,18 @@ int enqueue_predictor_plain(tw_handle* h, const int* tokens, const float* state_
 }
 
 // UpdatePredictorOutput for the work list the compaction kernel built (new slot, parent slot, token).
-void enqueue_predictor_slots(tw_handle* h, cudaStream_t st, int* launches) {
+// build_list: the compaction kernel did not run; the gather kernel derives the work list from the per-utterance
+// lists of new hypotheses itself (bf16 mode)
+void enqueue_predictor_slots(tw_handle* h, cudaStream_t st, int* launches, bool build_list = false, int B = 0) {
   if (h->pred_kind == TW_PRED_STATELESS) return;   // the joiner reads W_p emb[last token] from a table
   const HypState& hs = h->hs;
+  WorkListBuild wl{};
+  if (build_list) {
+    wl.B = B; wl.n_new = hs.n_new; wl.new_slot = hs.new_slot; wl.new_par = hs.new_par; wl.new_tok = hs.new_tok;
+    wl.pw_new = hs.pw_new; wl.pw_par = hs.pw_par; wl.pw_tok = hs.pw_tok; wl.n_out = hs.scalars + kScNPred;
+  }
   enqueue_predictor(h, hs.pw_tok, hs.slot_hc, hs.pw_par, hs.slot_hc, hs.pw_new, hs.slot_Pp,
-                    hs.scalars + kScNPred, h->R_max, st, launches);
+                    hs.scalars + kScNPred, h->R_max, st, launches, build_list ? &wl : nullptr);
 }
 
 // E = enc W_e^T for `rows` frames
