@@ -88,6 +88,9 @@ __global__ void __launch_bounds__(kThreads) hyp_init_kernel(HypState hs, const i
 }
 
 constexpr int kStepThreads = 512;   // 16 warps: one per hypothesis of list A
+constexpr int kSelCap = 64;         // survivors of a row's bound that are ranked directly
+
+__device__ __forceinline__ bool tok_better(float v1, int k1, float v2, int k2) { return v1 > v2 || (v1 == v2 && k1 < k2); }
 
 // Order-preserving integer image of a score: a < b as doubles <=> order_key(a) < order_key(b) as unsigned
 // integers (-0 counts as +0; scores are never NaN).  The ranking loops compare these instead of doubles.
@@ -107,6 +110,8 @@ __global__ void __launch_bounds__(kStepThreads) hyp_step_kernel(HypState hs) {
   __shared__ unsigned long long s_key[kMaxBeam * kMaxBeam];
   __shared__ unsigned long long s_nkey[32];
   __shared__ int s_nidx[32];
+  __shared__ float s_lm[kMaxBeam][32], s_sv[kMaxBeam][kSelCap];   // in-kernel selection: lane maxima, survivors of a row
+  __shared__ int s_sk[kMaxBeam][kSelCap], s_cnt[kMaxBeam];
   __shared__ int s_cursor, s_iters, s_nT0, s_Btop[kMaxBeam];     // per-utterance state fetched up front
   __shared__ double s_Btopls[kMaxBeam], s_tval[kMaxBeam];         // scores of B's old best / of the entries touched now
   __shared__ int s_sel[kMaxBeam];
@@ -134,6 +139,84 @@ __global__ void __launch_bounds__(kStepThreads) hyp_step_kernel(HypState hs) {
     s_carry[tid] = hs.carry[b * kMaxBeam + tid];
   }
   if (tid == 0) { hs.calls[b] += 1; hs.joins[b] += slen; }
+  if (hs.dnb_sel != nullptr) {
+    // ---- ChooseNBestExpansions, first stage, for the row of hypothesis `warp`: its N best tokens by delta_nb,
+    // order (value desc, token asc), straight into the candidate table of the second stage.
+    const int h = warp;
+    if (lane < kMaxBeam) {
+      s_abs[h * kMaxBeam + lane] = -INFINITY; s_ck[h * kMaxBeam + lane] = -1; s_key[h * kMaxBeam + lane] = order_key(-INFINITY);
+    }
+    __syncwarp();
+    if (h < H) {
+      const float* src = hs.dnb_sel + (long long)(r0 + h) * V;
+      const double base = hs.A_ls[b * kMaxBeam + h];
+      // a lower bound of the N-th best value: the N-th largest of the 32 lane maxima (distinct elements)
+      float lmax = 0.f;
+      for (int k = lane * 4; k < V; k += 128) {
+        const float4 v = __ldg(reinterpret_cast<const float4*>(src + k));
+        lmax = fmaxf(fmaxf(lmax, fmaxf(v.x, v.y)), fmaxf(v.z, v.w));
+      }
+      s_lm[h][lane] = lmax;
+      if (lane == 0) s_cnt[h] = 0;
+      __syncwarp();
+      int lrank = 0;
+#pragma unroll
+      for (int j = 0; j < 32; ++j) { const float o = s_lm[h][j]; lrank += (o > lmax || (o == lmax && j < lane)) ? 1 : 0; }
+      const unsigned who = __ballot_sync(0xffffffffu, lrank == N - 1);        // exactly one lane: the ranks are 0..31
+      const float bound = __shfl_sync(0xffffffffu, lmax, __ffs(who) - 1);
+      for (int k = lane * 4; k < V; k += 128) {
+        const float4 v4 = __ldg(reinterpret_cast<const float4*>(src + k));
+        const float vv[4] = {v4.x, v4.y, v4.z, v4.w};
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          if (vv[c] >= bound && vv[c] > 0.f) {
+            const int i = atomicAdd(&s_cnt[h], 1);
+            if (i < kSelCap) { s_sv[h][i] = vv[c]; s_sk[h][i] = k + c; }
+          }
+        }
+      }
+      __syncwarp();
+      const int ns = s_cnt[h];
+      if (ns <= kSelCap) {
+        for (int i = lane; i < ns; i += 32) {
+          const float v = s_sv[h][i]; const int k = s_sk[h][i];
+          int rank = 0;
+          for (int j = 0; j < ns; ++j) rank += tok_better(s_sv[h][j], s_sk[h][j], v, k) ? 1 : 0;
+          if (rank < N) {
+            const double sc = base + (double)__logf(v);
+            s_abs[h * kMaxBeam + rank] = sc; s_ck[h * kMaxBeam + rank] = k; s_key[h * kMaxBeam + rank] = order_key(sc);
+          }
+        }
+      } else {
+        // many ties at the bound: N rounds, each taking the best element after the previous pick in that order
+        float pv = INFINITY; int pk = -1;
+        for (int j = 0; j < N; ++j) {
+          float bv = 0.f; int bk = 0x7fffffff;
+          for (int k = lane * 4; k < V; k += 128) {
+            const float4 v4 = __ldg(reinterpret_cast<const float4*>(src + k));
+            const float vv[4] = {v4.x, v4.y, v4.z, v4.w};
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              const bool after = vv[c] < pv || (vv[c] == pv && k + c > pk);
+              if (vv[c] > 0.f && after && tok_better(vv[c], k + c, bv, bk)) { bv = vv[c]; bk = k + c; }
+            }
+          }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+            const int ok = __shfl_xor_sync(0xffffffffu, bk, o);
+            if (tok_better(ov, ok, bv, bk)) { bv = ov; bk = ok; }
+          }
+          if (!(bv > 0.f)) break;
+          if (lane == 0) {
+            const double sc = base + (double)__logf(bv);
+            s_abs[h * kMaxBeam + j] = sc; s_ck[h * kMaxBeam + j] = bk; s_key[h * kMaxBeam + j] = order_key(sc);
+          }
+          pv = bv; pk = bk;
+        }
+      }
+    }
+  }
   if (warp == 15) {
     // ring cursor, pass counter and the best-N set of list B as the previous pass left it: fetched now, by a
     // warp that has nothing to do in the search, so that the later phases find them in shared memory
@@ -234,7 +317,7 @@ __global__ void __launch_bounds__(kStepThreads) hyp_step_kernel(HypState hs) {
   }
   // ---- ChooseNBestExpansions, second stage: the N best (h, k) over the rows' candidate lists, in
   // float64; order (score desc, h asc, k asc).  The lists are sorted by (score desc, k asc).
-  if (tid < kMaxBeam * kMaxBeam) {
+  if (hs.dnb_sel == nullptr && tid < kMaxBeam * kMaxBeam) {
     const int h = tid / kMaxBeam, j = tid % kMaxBeam;
     const bool valid = h < H && j < hs.cand_n[r0 + h];
     s_abs[tid] = valid ? s_Als[h] + (double)hs.cand_v[(long long)(r0 + h) * kMaxBeam + j] : -INFINITY;

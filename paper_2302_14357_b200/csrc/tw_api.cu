@@ -225,6 +225,7 @@ int build_bf16(tw_handle* h) {
     }
   }
   h->hs.defer_rows = 0;
+  h->hs.dnb_sel = nullptr;
   h->hs_fused = h->hs;
   h->hs_fused.logp = nullptr; h->hs_fused.lse = nullptr; h->hs_fused.ldphi_d = nullptr; h->hs_fused.la_d = nullptr;
   if (h->mode == TW_MODE_BF16 && h->bf.fused_ok) {
@@ -233,6 +234,7 @@ int build_bf16(tw_handle* h) {
                 cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming) == cudaSuccess;
     if (!h->aux_ok) cudaGetLastError();
     h->hs_fused.defer_rows = h->aux_ok ? 1 : 0;
+    h->hs_fused.dnb_sel = h->hs.ldnb;            // the step's hyp_step_kernel picks the rows' best tokens itself
   }
   TW_CUDA(h, cudaGetLastError());
   return TW_OK;

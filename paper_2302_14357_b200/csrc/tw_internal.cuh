@@ -152,6 +152,9 @@ struct HypState {
   // row_ld and the clearing of n_new are left to the kernel that completes the new hypotheses' frame
   // distributions, which then runs beside the predictor kernels of the next pass
   int defer_rows;
+  // dnb_sel != nullptr: delta_nb [R][V] as plain probability ratios (0: no candidate); hyp_step_kernel then picks
+  // every row's N best tokens itself instead of reading cand_v / cand_k / cand_n
+  const float* dnb_sel;
   // list B of Algorithm 1 (hypotheses finished for this segment): [B][capB]
   int* B_slot; double* B_ls; unsigned long long* B_hash; int* B_len;
   int* B_top;    // [B][kMaxBeam] indices into list B of its best entries, best first
