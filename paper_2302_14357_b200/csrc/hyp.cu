@@ -99,7 +99,7 @@ __device__ __forceinline__ unsigned long long order_key(double x) {
   return (u >> 63) ? ~u : (u | 0x8000000000000000ull);
 }
 
-__global__ void __launch_bounds__(kStepThreads) hyp_step_kernel(HypState hs) {
+__global__ void __launch_bounds__(2 * kStepThreads) hyp_step_kernel(HypState hs) {
   __shared__ int s_nB, s_hasthr, s_nkeep;
   __shared__ int s_found[kMaxBeam], s_touched[kMaxBeam], s_carry[kMaxBeam];
   __shared__ double s_Als[kMaxBeam], s_Adone[kMaxBeam];
@@ -139,10 +139,18 @@ __global__ void __launch_bounds__(kStepThreads) hyp_step_kernel(HypState hs) {
     s_carry[tid] = hs.carry[b * kMaxBeam + tid];
   }
   if (tid == 0) { hs.calls[b] += 1; hs.joins[b] += slen; }
-  if (hs.dnb_sel != nullptr) {
-    // ---- ChooseNBestExpansions, first stage, for the row of hypothesis `warp`: its N best tokens by delta_nb,
+  // With in-kernel selection the CTA has 32 warps: warps 16..31 select (one row each) while warps 0..15 merge the
+  // blank expansions into list B and find the threshold; the two halves meet at the barrier before the ranking.
+  // Until then the merging half synchronises on a named barrier of its own.
+  const bool two_halves = hs.dnb_sel != nullptr;
+  auto sync_merge = [&]() {
+    if (two_halves) asm volatile("bar.sync 1, 512;" ::: "memory");
+    else __syncthreads();
+  };
+  if (two_halves && warp >= 16) {
+    // ---- ChooseNBestExpansions, first stage, for the row of hypothesis warp - 16: its N best tokens by delta_nb,
     // order (value desc, token asc), straight into the candidate table of the second stage.
-    const int h = warp;
+    const int h = warp - 16;
     if (lane < kMaxBeam) {
       s_abs[h * kMaxBeam + lane] = -INFINITY; s_ck[h * kMaxBeam + lane] = -1; s_key[h * kMaxBeam + lane] = order_key(-INFINITY);
     }
@@ -228,7 +236,7 @@ __global__ void __launch_bounds__(kStepThreads) hyp_step_kernel(HypState hs) {
       if (lane < nT) s_Btopls[lane] = hs.B_ls[bB + bt];       // before this pass's merges; touched entries are patched below
     }
   }
-  __syncthreads();
+  if (warp < 16) sync_merge();
 
   // ---- AddAndMerge, search: warp h looks for the tokens of A_h among the entries already in B.
   // (Entries of A are distinct sequences, so two of them never merge with each other.)
@@ -256,7 +264,7 @@ __global__ void __launch_bounds__(kStepThreads) hyp_step_kernel(HypState hs) {
     }
     if (lane == 0) { s_found[warp] = found; s_Alen[warp] = ln; }
   }
-  __syncthreads();
+  if (warp < 16) sync_merge();
   // ---- AddAndMerge, apply: sum into the matching entry or append (appends keep the order of A)
   if (tid < H) {
     const int h = tid;
@@ -282,7 +290,7 @@ __global__ void __launch_bounds__(kStepThreads) hyp_step_kernel(HypState hs) {
     s_nB = nB;
     hs.nB[b] = nB;
   }
-  __syncthreads();
+  if (warp < 16) sync_merge();
 
   // ---- ChooseNthScore: the best N of B are among the previous best N and the entries touched now
   if (warp == 0) {
@@ -581,7 +589,7 @@ void launch_hyp_init(const HypState& hs, const int* lengths, int B, int T, cudaS
   if (B > 0) hyp_init_kernel<<<B, kThreads, 0, st>>>(hs, lengths, T);
 }
 void launch_hyp_step(const HypState& hs, int B, cudaStream_t st) {
-  if (B > 0) launch_pdl(hyp_step_kernel, dim3(B), dim3(kStepThreads), 0, st, hs);
+  if (B > 0) launch_pdl(hyp_step_kernel, dim3(B), dim3(hs.dnb_sel ? 2 * kStepThreads : kStepThreads), 0, st, hs);
 }
 void launch_compact(const HypState& hs, int B, int T, cudaStream_t st) {
   launch_pdl(compact_kernel, dim3(1), dim3(1024), 0, st, hs, B, T);
