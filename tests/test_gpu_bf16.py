@@ -177,6 +177,30 @@ def test_decode_fused_equals_staged_bf16():
     assert sa["calls"] > 0 and np.all(a[3] == 0)
 
 
+def test_fused_path_selection_on_exact_ties():
+    """W_out = 0: all tokens of a row tie, far more than the direct ranking of the in-kernel selection holds,
+    so it runs on its round-by-round path; ties resolve to the smaller hypothesis index, then the smaller token."""
+    from paper_2302_14357_b200.binding import MODE_BF16, TwDecoder, weights_from_synth
+    cfg = _cfg(batch=5, T=9, V=256, J=64)
+    m = tw_synth.make_model(cfg)
+    m.W_out[:] = 0.0
+    m.b_out[:] = 0.0
+    enc, lens = tw_synth.make_encoder_batch(cfg)
+    lens[:] = [9, 4, 1, 7, 6]
+    N, S = 4, 3
+    dec = TwDecoder(weights_from_synth(m), N=N, S=S, mode=MODE_BF16, max_batch=5, max_T=9, max_iters_per_segment=3)
+    assert dec.set_fused(True)
+    tokens, olens, scores, status = [x.cpu().numpy() for x in dec.decode(enc, lens)[:4]]
+    om = oracle_model(m)
+    for b in range(5):
+        ref, st = tws.token_wise_beam_search(om, enc[b, :lens[b]].astype(np.float64), N, S, max_iters=3)
+        got = nbest_from_arrays(tokens, olens, scores, b)
+        assert [t for t, _ in got] == [t for t, _ in ref], (b, got, ref)
+        np.testing.assert_allclose([s for _, s in got], [s for _, s in ref], atol=2e-3)
+        assert status[b] == (4 if st.limit_hit else 0)
+    dec.close()
+
+
 def _top1_agreement(cfg, S, batch, T):
     from paper_2302_14357_b200.binding import MODE_BF16, TwDecoder, weights_from_synth
     m = tw_synth.make_model(cfg)
