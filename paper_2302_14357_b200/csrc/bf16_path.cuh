@@ -39,8 +39,9 @@ struct GemmBf16Params {
 int make_tmap_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint64_t K, uint32_t box_rows);
 int gemm_bf16_setup();
 // tmB128 / tmB256: maps of the same B matrix with 128- and 256-row boxes
+// tmB64 (optional): a map with 64-row boxes, used for small problems without an epilogue fusion
 void launch_gemm_bf16(const CUtensorMap& tmA, const CUtensorMap& tmB128, const CUtensorMap& tmB256,
-                      const GemmBf16Params& p, cudaStream_t st);
+                      const GemmBf16Params& p, cudaStream_t st, const CUtensorMap* tmB64 = nullptr);
 
 // LSTM gate GEMM (epi == 1) as a single wave of one tile per CTA when 128 x 256 tiles would need a second,
 // nearly empty wave; returns false (nothing launched) when the shape does not call for it.

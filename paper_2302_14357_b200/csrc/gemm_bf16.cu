@@ -20,7 +20,7 @@ constexpr int kThreadsGemm = 64 + 32 * kEpiWarps;
 
 template <int BN>
 struct Cfg {
-  static constexpr int kStages = (BN == 256) ? 4 : 6;
+  static constexpr int kStages = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
   static constexpr uint32_t kABytes = BM * BK * 2, kBBytes = BN * BK * 2;
   static constexpr size_t kSmem = (size_t)kStages * (kABytes + kBBytes) + 1024 + 256;
 };
@@ -476,6 +476,8 @@ int gemm_bf16_setup() {
   cudaError_t e2 = cudaFuncSetAttribute(gemm_bf16_kernel<128, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<128>::kSmem);
   cudaError_t e3 = cudaFuncSetAttribute(gemm_bf16_kernel<256, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<256>::kSmem);
   cudaError_t e4 = cudaFuncSetAttribute(gemm_bf16_kernel<128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<128>::kSmem);
+  cudaError_t e6 = cudaFuncSetAttribute(gemm_bf16_kernel<64, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<64>::kSmem);
+  if (e6 != cudaSuccess) return TW_ERR_CUDA;
   cudaError_t e5 = cudaFuncSetAttribute(gemm_lstm_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kWideSmem);
   return (e1 == cudaSuccess && e2 == cudaSuccess && e3 == cudaSuccess && e4 == cudaSuccess && e5 == cudaSuccess) ? TW_OK : TW_ERR_CUDA;
 }
@@ -505,7 +507,7 @@ bool launch_gemm_lstm_wide(const CUtensorMap& tmA, const CUtensorMap& tmB64, con
 }
 
 void launch_gemm_bf16(const CUtensorMap& tmA, const CUtensorMap& tmB128, const CUtensorMap& tmB256,
-                      const GemmBf16Params& p, cudaStream_t st) {
+                      const GemmBf16Params& p, cudaStream_t st, const CUtensorMap* tmB64) {
   if (p.M <= 0 || p.N <= 0) return;
   const int num_sms = sm_count();
   const int mt = (p.M + BM - 1) / BM;
@@ -515,6 +517,11 @@ void launch_gemm_bf16(const CUtensorMap& tmA, const CUtensorMap& tmB128, const C
     const int grid = (int)((long long)mt * nt256 < num_sms ? mt * nt256 : num_sms);
     if (p.epi == 1) launch_pdl(gemm_bf16_kernel<256, 1>, dim3(grid), dim3(kThreadsGemm), Cfg<256>::kSmem, st, tmA, tmB256, p);
     else launch_pdl(gemm_bf16_kernel<256, 0>, dim3(grid), dim3(kThreadsGemm), Cfg<256>::kSmem, st, tmA, tmB256, p);
+  } else if (tmB64 != nullptr && p.epi == 0 && (long long)mt * nt128 * 4 <= (long long)num_sms * 3) {
+    // few tiles and a short K loop each: 64-column tiles put twice as many SMs to work
+    const long long tiles = (long long)mt * ((p.N + 63) / 64);
+    const int grid = (int)(tiles < num_sms ? tiles : num_sms);
+    launch_pdl(gemm_bf16_kernel<64, 0>, dim3(grid), dim3(kThreadsGemm), Cfg<64>::kSmem, st, tmA, *tmB64, p);
   } else {
     const long long tiles = (long long)mt * nt128;
     const int grid = (int)(tiles < num_sms ? tiles : num_sms);

@@ -59,7 +59,7 @@ void gemm_bf16(tw_handle* h, const Bf16Mat& A, const Bf16Mat& B, const int* M_de
                const int* add_idx = nullptr, long long ld_add = 0) {
   GemmBf16Params p{M_dev, M, (int)B.rows, (int)A.K, C, oidx, ldC, bias, h->bf.err};
   p.addend = addend; p.add_idx = add_idx; p.ld_add = ld_add;
-  launch_gemm_bf16(A.as_A, B.as_B128, B.as_B256, p, st);
+  launch_gemm_bf16(A.as_A, B.as_B128, B.as_B256, p, st, &B.as_B64);
 }
 
 // UpdatePredictorOutput for n hypotheses: one predictor step on tok[i] from the state at row
