@@ -205,10 +205,22 @@ int build_bf16(tw_handle* h) {
     }
   }
   // fused joiner: needs S frames of a hypothesis inside one warp and V split into 256-column CTAs
-  if (fused_joiner_eligible(h->S, h->V, h->J)) {
-    h->bf.CL = h->V / 256;
+  h->bf.Vp = (h->V + 255) / 256 * 256;
+  if (fused_joiner_eligible(h->S, h->bf.Vp, h->J)) {
+    h->bf.CL = h->bf.Vp / 256;
     int s = fused_joiner_setup(h->bf.CL, h->S, &h->bf.max_clusters);
     if (s == TW_OK) {
+      if (h->bf.Vp == h->V) {
+        h->bf.W_out_pad = h->bf.W_out; h->bf.bias_pad = h->b_out; h->bf.ldnb_pad = h->hs.ldnb;
+      } else {
+        TW_TRY(make_bf16_mat(h, &h->bf.W_out_pad, nullptr, h->bf.Vp, h->J, false, true));      // zero rows
+        launch_f32_to_bf16(h->W_out, h->bf.W_out_pad.ptr, (long long)h->V * h->J, 0);
+        std::vector<float> bias((size_t)h->bf.Vp, -1e30f);
+        TW_CUDA(h, cudaMemcpy(bias.data(), h->b_out, (size_t)h->V * sizeof(float), cudaMemcpyDeviceToHost));
+        TW_TRY(dev_alloc(h, &h->bf.bias_pad, (size_t)h->bf.Vp));
+        TW_CUDA(h, cudaMemcpy(h->bf.bias_pad, bias.data(), (size_t)h->bf.Vp * sizeof(float), cudaMemcpyHostToDevice));
+        TW_TRY(dev_alloc(h, &h->bf.ldnb_pad, (size_t)h->R_max * h->bf.Vp));
+      }
       // |z| <= max_k (|W_out[k, :]|_1 + |b_out[k]|) because |tanh| <= 1: small enough => sum exp(z) needs no max
       float* bound_dev = nullptr; float bound = 0.f;
       TW_TRY(dev_alloc(h, &bound_dev, (size_t)1));
@@ -234,7 +246,8 @@ int build_bf16(tw_handle* h) {
                 cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming) == cudaSuccess;
     if (!h->aux_ok) cudaGetLastError();
     h->hs_fused.defer_rows = h->aux_ok ? 1 : 0;
-    h->hs_fused.dnb_sel = h->hs.ldnb;            // the step's hyp_step_kernel picks the rows' best tokens itself
+    h->hs_fused.dnb_sel = h->bf.ldnb_pad;        // the step's hyp_step_kernel picks the rows' best tokens itself
+    h->hs_fused.V = h->bf.Vp;                    // row pitch of delta_nb there (padding columns hold 0)
   }
   TW_CUDA(h, cudaGetLastError());
   return TW_OK;
@@ -395,17 +408,17 @@ int enqueue_joiner_fused(tw_handle* h, const JoinerRows& rows, const float* ld_o
     launch_joiner_A_tiled(rows, h->bf.A_tiled.ptr, st);
   }
   if (mark_fn) mark_fn(h, 3, st);       // operand preparation is booked with the elementwise stages
-  if (ldnb == nullptr) ldnb = h->hs.ldnb;
+  if (ldnb == nullptr) ldnb = h->bf.ldnb_pad;   // a caller's buffer has V columns: only with an unpadded vocabulary
   FusedJoinerParams fp{};
-  fp.R_dev = rows.R_dev; fp.R_max = rows.R_max; fp.S = rows.S; fp.V = rows.V; fp.K = rows.J; fp.blank = h->blank;
-  fp.CL = h->bf.CL; fp.no_max = h->bf.no_max ? 1 : 0; fp.bias = h->b_out; fp.ld_old = ld_old; fp.row_slen = rows.row_slen;
+  fp.R_dev = rows.R_dev; fp.R_max = rows.R_max; fp.S = rows.S; fp.V = h->bf.Vp; fp.K = rows.J; fp.blank = h->blank;
+  fp.CL = h->bf.CL; fp.no_max = h->bf.no_max ? 1 : 0; fp.bias = h->bf.bias_pad; fp.ld_old = ld_old; fp.row_slen = rows.row_slen;
   fp.ldphi = ldphi; fp.la = la; fp.lse = h->bf.lse; fp.ldnb = ldnb; fp.err = h->bf.err;
-  TW_TRY(launch_fused_joiner(h->bf.A_tiled.as_A, h->bf.W_out.as_B256, fp, h->bf.max_clusters, st));
+  TW_TRY(launch_fused_joiner(h->bf.A_tiled.as_A, h->bf.W_out_pad.as_B256, fp, h->bf.max_clusters, st));
   if (mark_fn) mark_fn(h, 2, st);       // the fused kernel alone
   *launches += 2;
   if (cand.n != nullptr) {      // ChooseNBestExpansions, first stage: the rows' N best tokens
     ScanSelectArgs a{};
-    a.R_dev = rows.R_dev; a.R_max = rows.R_max; a.S = rows.S; a.V = rows.V; a.blank = h->blank;
+    a.R_dev = rows.R_dev; a.R_max = rows.R_max; a.S = rows.S; a.V = h->bf.Vp; a.blank = h->blank;
     a.cand = cand; a.dnb_in = ldnb; a.dnb_linear = 1;
     launch_scan_select(a, true, st);
     *launches += 1;

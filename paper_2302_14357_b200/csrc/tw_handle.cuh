@@ -41,6 +41,13 @@ struct tw_handle {
     // fused joiner + softmax + Eq. 3-7 + selection (logits stay in tensor memory)
     bool fused_ok = false, fused_on = false, no_max = false;
     int CL = 0, max_clusters = 0;
+    // The fused kernel splits the vocabulary into 256-column CTAs.  A vocabulary that is not a multiple of 256 is
+    // padded for it: Vp columns, the added rows of W_out zero and their bias -1e30 (probability 0, never a
+    // candidate).  Vp == V: the padded objects below are the plain ones.
+    int Vp = 0;
+    tw::Bf16Mat W_out_pad;
+    float* bias_pad = nullptr;
+    float* ldnb_pad = nullptr;                            // [R_max, Vp]
     tw::Bf16Mat A_tiled;                                  // A operand in the fused kernel's tile layout
     float* lse = nullptr;                                 // [R_max, S]
   } bf;

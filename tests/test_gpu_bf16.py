@@ -177,6 +177,34 @@ def test_decode_fused_equals_staged_bf16():
     assert sa["calls"] > 0 and np.all(a[3] == 0)
 
 
+@pytest.mark.parametrize("V,act", [(501, "relu"), (300, "tanh"), (1000, "tanh")])
+def test_fused_path_with_padded_vocabulary(V, act):
+    """A vocabulary that is not a multiple of 256 is padded for the fused kernel (zero weight rows, bias -1e30):
+    same top-1 as the oracle, same N-best as the staged kernels, no padding token ever returned."""
+    from paper_2302_14357_b200.binding import MODE_BF16, TwDecoder, weights_from_synth
+    cfg = _cfg(batch=6, T=36, V=V).with_(joiner_act=act)
+    m = tw_synth.make_model(cfg)
+    enc, lens = tw_synth.make_encoder_batch(cfg)
+    N, S = 4, 3
+    dec = TwDecoder(weights_from_synth(m), N=N, S=S, mode=MODE_BF16, max_batch=6, max_T=36, joiner_act=act)
+    assert dec.set_fused(True) and dec.stats()["fused_on"] == 1
+    a = [x.cpu().numpy() for x in dec.decode(enc, lens)[:4]]
+    assert dec.set_fused(False)
+    b = [x.cpu().numpy() for x in dec.decode(enc, lens)[:4]]
+    assert a[0].max() < V and np.all(a[3] == 0)
+    same = sum(int(np.array_equal(a[0][u, 0], b[0][u, 0])) for u in range(6))
+    assert same >= 5
+    np.testing.assert_allclose(a[2][:, 0], b[2][:, 0], atol=0.05)
+    om = oracle_model(m)
+    agree = 0
+    for u in range(6):
+        ref, _ = tws.token_wise_beam_search(om, enc[u, :lens[u]].astype(np.float64), N, S, max_iters=4 * S + 16)
+        got = nbest_from_arrays(a[0], a[1], a[2], u)
+        agree += int(got[0][0] == ref[0][0])
+    assert agree >= 5
+    dec.close()
+
+
 def test_fused_path_selection_on_exact_ties():
     """W_out = 0: all tokens of a row tie, far more than the direct ranking of the in-kernel selection holds,
     so it runs on its round-by-round path; ties resolve to the smaller hypothesis index, then the smaller token."""
@@ -207,7 +235,7 @@ def _top1_agreement(cfg, S, batch, T):
     enc, lens = tw_synth.make_encoder_batch(cfg, batch)
     enc, lens = np.ascontiguousarray(enc[:, :T]), np.minimum(lens, T)
     dec = TwDecoder(weights_from_synth(m), N=cfg.N, S=S, mode=MODE_BF16, max_batch=batch, max_T=T)
-    assert dec.set_fused(True) == (cfg.V % 256 == 0)       # V = 501 runs the staged kernels
+    assert dec.set_fused(True)                             # V = 501 is padded to 512 columns for the fused kernel
     tokens, olens, scores, status, rc = [x.cpu().numpy() if hasattr(x, "cpu") else x for x in dec.decode(enc, lens)]
     om = oracle_model(m)
     agree, gaps = 0, []
