@@ -260,11 +260,12 @@ int tw_joiner_expand_noalloc(const float* W_out, const float* b_out, int32_t J, 
                              int32_t G, int32_t R, float* out_ldphi, float* out_ldnb, float* out_la,
                              void* stream);
 
-/* TW_MODE_BF16 only: switches between the fused joiner (joiner, softmax, Eq. 3-7 and the first stage
- * of ChooseNBestExpansions in one kernel, logits kept in tensor memory; available when S <= 32 and V is a
- * multiple of 256 up to 4096, and the default for S in {1..5, 8, 10}) and the staged kernels that pass the logits through
- * device memory.  Both compute the same quantities.  TW_ERR_STATE if the fused kernel is not
- * available for this handle. */
+/* TW_MODE_BF16 only: switches between the fused joiner (joiner, softmax and Eq. 3-7 in one kernel, logits
+ * kept in tensor memory; available when S <= 32 and V <= 4096, a vocabulary that is not a multiple of 256
+ * being padded internally with columns of probability 0; the default for S in {1..5, 8, 10}) and the
+ * staged kernels that pass the logits through device memory.  Both compute the same quantities.
+ * tw_joiner_expand uses the fused kernel only with an unpadded vocabulary (its delta_nb rows have V
+ * columns).  TW_ERR_STATE if the fused kernel is not available for this handle. */
 int tw_set_fused(tw_handle* h, int on);
 
 /* tw_decode replays its step body (16 device steps) as a CUDA graph, captured once per batch shape, on
