@@ -140,7 +140,11 @@ int tw_decode(tw_handle* h, const float* enc, const int32_t* lengths, int32_t B,
               void* stream);
 
 /* Same as tw_decode with HOST buffers: copies the inputs to the device, decodes, copies the four
- * outputs back.  All copies are on `stream`; synchronises before returning. */
+ * outputs back; synchronises before returning.  For batches decoded in one piece and T >= 16 S the
+ * frames are uploaded in three time chunks on a stream of the handle's own (ordered after `stream`)
+ * and each chunk is decoded, as a streaming push, while the next one is on its way; the result is
+ * the same as tw_decode's.  Pinned host memory is what makes the upload asynchronous.  Must not be
+ * called while a streaming session is open on the handle. */
 int tw_decode_host(tw_handle* h, const float* host_enc, const int32_t* host_lengths, int32_t B,
                    int32_t T, int32_t* host_out_tokens, int32_t* host_out_lens,
                    double* host_out_scores, int32_t* host_out_status, void* stream);

@@ -497,6 +497,8 @@ int tw_destroy(tw_handle* h) {
   if (h->graph_exec) cudaGraphExecDestroy(h->graph_exec);
   if (h->ev_order) cudaEventDestroy(h->ev_order);
   if (h->ev_poll) cudaEventDestroy(h->ev_poll);
+  for (cudaEvent_t e : h->ev_chunk) if (e) cudaEventDestroy(e);
+  if (h->copy_stream) cudaStreamDestroy(h->copy_stream);
   if (h->ev_fork) cudaEventDestroy(h->ev_fork);
   if (h->ev_join) cudaEventDestroy(h->ev_join);
   if (h->aux_stream) cudaStreamDestroy(h->aux_stream);

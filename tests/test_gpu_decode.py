@@ -164,3 +164,26 @@ def test_decode_host_equals_device_decode():
     c = dec.decode_host(enc, lens)[:4]
     for x, y in zip(b, c):
         np.testing.assert_array_equal(x, y)
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_decode_host_chunked_upload_ragged_batch(mode):
+    """tw_decode_host uploads in time chunks and decodes each as it arrives: same result as tw_decode on device
+    buffers, for ragged lengths (empty, one frame, full), and also when a length is out of range (which takes the
+    plain path and reports the utterance)."""
+    from paper_2302_14357_b200.binding import TwDecoder, weights_from_synth
+    cfg = tw_synth.WorkloadConfig("h", 6, 64, (0, 64), 64, "lstm", 32, 1, 32, 64, 256, 2.0, 3, (3,), "bf16" if mode else "f32", 11)
+    m = tw_synth.make_model(cfg)
+    enc, lens = tw_synth.make_encoder_batch(cfg)
+    lens[:] = [64, 0, 1, 37, 50, 63]
+    dec = TwDecoder(weights_from_synth(m), N=3, S=3, mode=mode, max_batch=6, max_T=64)
+    a = [x.cpu().numpy() for x in dec.decode(enc, lens)[:4]]
+    b = dec.decode_host(enc, lens)[:4]
+    for x, y in zip(a, b):
+        np.testing.assert_array_equal(x, y)
+    bad = lens.copy()
+    bad[3] = 99
+    c = dec.decode_host(enc, bad)
+    assert c[3][3] == 1 and c[3][0] == 0           # TW_ERR_ARG for that utterance only
+    np.testing.assert_array_equal(c[0][0], a[0][0])
+    dec.close()
