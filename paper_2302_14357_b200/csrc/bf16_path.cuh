@@ -108,6 +108,9 @@ void launch_logit_bound(const __nv_bfloat16* W, const float* bias, int V, int J,
 // in place: x -> log x (log 0 = -inf), n elements
 void launch_log_inplace(float* x, long long n, cudaStream_t st);
 void launch_joiner_A_tiled(const JoinerRows& rows, __nv_bfloat16* A, cudaStream_t st);
+// the same for the rows of a decode step (utterance b's rows are row_off[b] .. + nA[b] - 1, all on one segment)
+void launch_joiner_A_tiled_utt(const JoinerRows& rows, const int* row_off, const int* nA, int B, __nv_bfloat16* A,
+                               cudaStream_t st);
 int launch_fused_joiner(const CUtensorMap& tmA, const CUtensorMap& tmB256, const FusedJoinerParams& p,
                         int max_clusters, cudaStream_t st);
 // adds log J(t, parent row, token) to A_ld of the hypotheses created in this step

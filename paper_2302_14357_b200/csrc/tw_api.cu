@@ -402,10 +402,11 @@ void enqueue_scan(tw_handle* h, const JoinerRows& rows, const float* ld_old, flo
 // Fused path: joiner, softmax, Eq. 3-7 and per-row candidates with the logits kept in tensor memory
 int enqueue_joiner_fused(tw_handle* h, const JoinerRows& rows, const float* ld_old, float* ldphi, float* ldnb,
                          float* la, const CandOut& cand, cudaStream_t st, int* launches, StageMarkFn mark_fn,
-                         bool plain_first) {
+                         bool plain_first, int utt_B) {
   {
     PdlScope first(plain_first ? false : g_pdl_on);
-    launch_joiner_A_tiled(rows, h->bf.A_tiled.ptr, st);
+    if (utt_B > 0) launch_joiner_A_tiled_utt(rows, h->hs.row_off, h->hs.nA, utt_B, h->bf.A_tiled.ptr, st);
+    else launch_joiner_A_tiled(rows, h->bf.A_tiled.ptr, st);
   }
   if (mark_fn) mark_fn(h, 3, st);       // operand preparation is booked with the elementwise stages
   if (ldnb == nullptr) ldnb = h->bf.ldnb_pad;   // a caller's buffer has V columns: only with an unpadded vocabulary
