@@ -260,3 +260,12 @@ def test_decode_bf16_config_shapes_top1(name, S, batch, T):
     print("%s bf16 top-1 agreement %.2f, max top-1 score gap %.3g" % (name, rate, gap))
     assert rate >= 0.5 and gap < 1.0
     assert st["calls"] > 0
+
+
+@pytest.mark.parametrize("N", [1, 2])
+def test_decode_bf16_paper_shape_small_beams(N):
+    """The paper's tables also use beams of 1 and 2: greedy-sized lists on the paper-shaped workload."""
+    cfg = tw_synth.get_config("p1").with_(N=N)
+    rate, gap, st = _top1_agreement(cfg, 3, 4, 60)
+    assert rate >= 0.5 and gap < 1.0
+    assert st["calls"] > 0 and st["fused_on"] == 1
