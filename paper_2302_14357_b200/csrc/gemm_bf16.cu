@@ -502,7 +502,8 @@ bool launch_gemm_lstm_wide(const CUtensorMap& tmA, const CUtensorMap& tmB64, con
   if (n_split < 1) return false;
   const int units = p.N >> 5;
   if (((units + n_split - 1) / n_split) * 32 > kWideMaxBN) return false;
-  launch_pdl(gemm_lstm_wide_kernel, dim3(mt * n_split), dim3(kThreadsWide), kWideSmem, st, tmA, tmB64, tmB32, p);
+  // one CTA per SM: the kernel splits the columns of each row tile over floor(grid / row tiles of this launch) CTAs
+  launch_pdl(gemm_lstm_wide_kernel, dim3(num_sms), dim3(kThreadsWide), kWideSmem, st, tmA, tmB64, tmB32, p);
   return true;
 }
 
