@@ -42,13 +42,18 @@ __global__ void gather_parents_bf16_kernel(GatherParents g, const int* n_dev, in
     const int b0 = threadIdx.x * per, b1 = min(b0 + per, B);
     int mine = 0;
     for (int b = b0; b < b1; ++b) mine += g.wl.n_new[b];
-    s_run[threadIdx.x] = mine;
+    // exclusive scan of the 128 run sums: shuffles inside the warps, then the four warp totals
+    __shared__ int s_wtot[4];
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    int inc = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += v; }
+    if (lane == 31) s_wtot[wid] = inc;
     __syncthreads();
-    if (threadIdx.x == 0) {
-      int acc = 0;
-      for (int i = 0; i < (int)blockDim.x; ++i) { const int v = s_run[i]; s_run[i] = acc; acc += v; }
-      s_total = acc;
-    }
+    int before = 0;
+    for (int w = 0; w < wid; ++w) before += s_wtot[w];
+    s_run[threadIdx.x] = before + inc - mine;
+    if (threadIdx.x == blockDim.x - 1) s_total = before + inc;
     __syncthreads();
     n = s_total;
     if (r == 0 && l == 0 && threadIdx.x == 0) *g.wl.n_out = n;
