@@ -122,22 +122,24 @@ __global__ void __launch_bounds__(2 * kStepThreads) hyp_step_kernel(HypState hs)
   pdl_trigger();
   const int b = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  // every first-round load is issued before the early exit below, so that none of them waits for H
   const int H = hs.nA[b];
-  if (H == 0) return;                       // idle (finished) utterance
-  const int N = hs.N, S = hs.S, V = hs.V;
   const int r0 = hs.row_off[b];
   const int slen = hs.slen[b];
   const int nB0 = hs.nB[b];
+  double ld_Als = 0.0, ld_Adone = -INFINITY;
+  int ld_Aslot = 0, ld_carry = -1;
+  if (tid < kMaxBeam) {                     // all kMaxBeam entries of the lists; those past H are never used
+    ld_Als = hs.A_ls[b * kMaxBeam + tid]; ld_Aslot = hs.A_slot[b * kMaxBeam + tid];
+    if (hs.mono) ld_Adone = hs.A_done[b * kMaxBeam + tid];
+    ld_carry = hs.carry[b * kMaxBeam + tid];
+  }
+  if (H == 0) return;                       // idle (finished) utterance
+  const int N = hs.N, S = hs.S, V = hs.V;
   const long long bB = (long long)b * hs.capB;
   const long long bS = (long long)b * hs.capSlot;
 
-  if (tid < kMaxBeam) {
-    if (tid < H) {
-      s_Als[tid] = hs.A_ls[b * kMaxBeam + tid]; s_Aslot[tid] = hs.A_slot[b * kMaxBeam + tid];
-      s_Adone[tid] = hs.mono ? hs.A_done[b * kMaxBeam + tid] : -INFINITY;
-    }
-    s_carry[tid] = hs.carry[b * kMaxBeam + tid];
-  }
+  if (tid < kMaxBeam) { s_Als[tid] = ld_Als; s_Aslot[tid] = ld_Aslot; s_Adone[tid] = ld_Adone; s_carry[tid] = ld_carry; }
   if (tid == 0) { hs.calls[b] += 1; hs.joins[b] += slen; }
   // With in-kernel selection the CTA has 32 warps: warps 16..31 select (one row each) while warps 0..15 merge the
   // blank expansions into list B and find the threshold; the two halves meet at the barrier before the ranking.
