@@ -47,7 +47,7 @@ void launch_gemm_bf16(const CUtensorMap& tmA, const CUtensorMap& tmB128, const C
 // nearly empty wave; returns false (nothing launched) when the shape does not call for it.
 // tmB64 / tmB32: maps of B with 64- and 32-row boxes
 bool launch_gemm_lstm_wide(const CUtensorMap& tmA, const CUtensorMap& tmB64, const CUtensorMap& tmB32,
-                           const GemmBf16Params& p, cudaStream_t st);
+                           const GemmBf16Params& p, cudaStream_t st, const CUtensorMap* tmB16 = nullptr);
 
 // A bf16 matrix with its tensor maps
 struct Bf16Mat {
@@ -55,7 +55,7 @@ struct Bf16Mat {
   long long rows = 0, K = 0;
   CUtensorMap as_A;            // box 128 rows
   CUtensorMap as_B128, as_B256;
-  CUtensorMap as_B64, as_B32;
+  CUtensorMap as_B64, as_B32, as_B16;
 };
 
 // elementwise helpers ---------------------------------------------------------------------------

@@ -50,6 +50,7 @@ int make_bf16_mat(tw_handle* h, Bf16Mat* m, const float* src, long long rows, lo
     TW_TRY(make_tmap_bf16(&m->as_B256, m->ptr, rows, K, 256));
     TW_TRY(make_tmap_bf16(&m->as_B64, m->ptr, rows, K, 64));
     TW_TRY(make_tmap_bf16(&m->as_B32, m->ptr, rows, K, 32));
+    TW_TRY(make_tmap_bf16(&m->as_B16, m->ptr, rows, K, 16));
   }
   return TW_OK;
 }
@@ -93,7 +94,7 @@ void enqueue_predictor(tw_handle* h, const int* tok, const float* hc_in, const i
       p.epi = 1;
       p.lstm = LstmEpi{hc_in, idx_in, hc_out, idx_out, L, l, Hd,
                        (l + 1 < L) ? h->bf.X[l + 1].ptr : h->bf.Htop.ptr, (l + 1 < L) ? 2LL * Hd : (long long)Hd};
-      if (!launch_gemm_lstm_wide(h->bf.X[l].as_A, h->bf.W_cat[l].as_B64, h->bf.W_cat[l].as_B32, p, st))
+      if (!launch_gemm_lstm_wide(h->bf.X[l].as_A, h->bf.W_cat[l].as_B64, h->bf.W_cat[l].as_B32, p, st, &h->bf.W_cat[l].as_B16))
         launch_gemm_bf16(h->bf.X[l].as_A, h->bf.W_cat[l].as_B128, h->bf.W_cat[l].as_B256, p, st);
     }
     gemm_bf16(h, h->bf.Htop, h->bf.W_p, n_dev, n_max, Pp_out, idx_out, h->J, nullptr, st);

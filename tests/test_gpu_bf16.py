@@ -293,3 +293,34 @@ def test_repeated_decodes_are_bit_identical():
     for x, y in zip(got, ref):
         np.testing.assert_array_equal(x, y)
     dec.close()
+
+
+def test_cta_pair_gate_gemm_matches_single_cta_kernel(tmp_path):
+    """TW_GEMM_PAIRS=1 runs the LSTM gate GEMMs on CTA pairs (tcgen05 cta_group::2).  The switch is read once per
+    process, so the pair run is a child process; both runs accumulate K in the same order."""
+    import os, subprocess, sys
+    code = """
+import sys, numpy as np, tw_synth
+sys.path.insert(0, 'tests')
+from paper_2302_14357_b200.binding import MODE_BF16, TwDecoder, weights_from_synth
+cfg = tw_synth.WorkloadConfig('b', 4, 30, (15, 30), 64, 'lstm', 64, 2, 1024, 128, 256, 3.0, 4, (3,), 'bf16', 3)
+m = tw_synth.make_model(cfg)
+R = 1200
+dec = TwDecoder(weights_from_synth(m), N=4, S=2, mode=MODE_BF16, max_batch=R // 4, max_T=30)
+rng = np.random.default_rng(4)
+tokens = rng.integers(0, cfg.V, size=R).astype(np.int32)
+state = (rng.standard_normal((R, 2, 2, 1024)) * 0.5).astype(np.float32)
+out, Pp = dec.predictor_step(tokens, state)
+np.savez(sys.argv[1], out=out.cpu().numpy(), Pp=Pp.cpu().numpy())
+"""
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    res = {}
+    for name, flag in (("single", "0"), ("pair", "1")):
+        path = str(tmp_path / (name + ".npz"))
+        env = dict(os.environ, TW_GEMM_PAIRS=flag, PYTHONPATH=root)
+        r = subprocess.run([sys.executable, "-c", code, path], env=env, cwd=root, capture_output=True, text=True, timeout=300)
+        assert r.returncode == 0, r.stderr[-2000:]
+        res[name] = np.load(path)
+    assert np.all(np.isfinite(res["pair"]["out"]))
+    np.testing.assert_allclose(res["pair"]["out"], res["single"]["out"], rtol=0, atol=1e-5)
+    np.testing.assert_allclose(res["pair"]["Pp"], res["single"]["Pp"], rtol=0, atol=1e-4)
