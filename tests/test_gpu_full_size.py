@@ -13,6 +13,10 @@ pytestmark = pytest.mark.gpu
 def _decode(cfg, S, mode, T=None):
     from paper_2302_14357_b200.binding import TwDecoder, weights_from_synth
     m = tw_synth.make_model(cfg)
+    if T is not None and cfg.batch * cfg.T > 200000:
+        # the 512-utterance workload: the same model and batch size with frames drawn for T frames only (its full
+        # input is 2 GB), lengths ragged and no multiple of S
+        cfg = cfg.with_(T=T, len_range=(T - 30, T))
     enc, lens = tw_synth.make_encoder_batch(cfg)
     if T is not None:
         enc, lens = np.ascontiguousarray(enc[:, :T]), np.minimum(lens, T)
@@ -23,7 +27,8 @@ def _decode(cfg, S, mode, T=None):
     return m, enc, lens, out, st
 
 
-@pytest.mark.parametrize("name,S,sample,T", [("c2", 3, (0, 37), None), ("c1", 5, (3, 30), None), ("c3", 3, (5, 90), 240)])
+@pytest.mark.parametrize("name,S,sample,T", [("c2", 3, (0, 37), None), ("c1", 5, (3, 30), None), ("c3", 3, (5, 90), 240),
+                                             ("c4", 10, (7, 300), 100)])
 def test_full_batch_fp32_sampled_utterances(name, S, sample, T):
     cfg = tw_synth.get_config(name)
     m, enc, lens, (tokens, olens, scores, status), st = _decode(cfg, S, 0, T)
@@ -53,4 +58,34 @@ def test_full_batch_bf16_c3_top1_sampled():
         agree += got[0][0] == ref[0][0]
         assert abs(got[0][1] - ref[0][1]) < 1.0
     print("c3 bf16 top-1 agreement on sampled utterances: %d/%d" % (agree, len(sample)))
+    assert agree >= 2
+
+
+def test_full_batch_bf16_c4_two_lanes_ragged_sampled():
+    """The 512-utterance stress shape (S = 10) in the configuration that is timed: bf16 fused joiner, the batch
+    split in two concurrent halves.  Ragged lengths that are no multiple of S; one sampled utterance per half and
+    one at the seam against the oracle (top-1), and every utterance against the same batch decoded in one piece."""
+    from paper_2302_14357_b200.binding import TwDecoder, weights_from_synth
+    S, T = 10, 120
+    cfg = tw_synth.get_config("c4").with_(T=T, len_range=(T - 30, T))     # the model and batch size, shorter input
+    m = tw_synth.make_model(cfg)
+    enc, lens = tw_synth.make_encoder_batch(cfg)
+    dec = TwDecoder(weights_from_synth(m), N=cfg.N, S=S, mode=1, max_batch=cfg.batch, max_T=T)
+    tokens, olens, scores, status = [x.cpu().numpy() for x in dec.decode(enc, lens)[:4]]
+    st = dec.stats()
+    dec.set_lanes(False)
+    one_piece = [x.cpu().numpy() for x in dec.decode(enc, lens)[:4]]
+    dec.close()
+    for x, y in zip((tokens, olens, scores, status), one_piece):
+        np.testing.assert_array_equal(x, y)
+    assert st["limit_hits"] == 0 and np.all(status == 0)
+    assert st["frames"] == int(lens.sum()) and np.all(np.diff(scores, axis=1) <= 0)
+    om = oracle_model(m)
+    agree, sample = 0, (7, 255, 300)
+    for b in sample:
+        got = nbest_from_arrays(tokens, olens, scores, b)
+        ref, _ = tws.token_wise_beam_search(om, enc[b, :lens[b]], cfg.N, S, max_iters=4 * S + 16)
+        agree += got[0][0] == ref[0][0]
+        assert abs(got[0][1] - ref[0][1]) < 1.0
+    print("c4 bf16 top-1 agreement on sampled utterances: %d/%d" % (agree, len(sample)))
     assert agree >= 2
