@@ -75,6 +75,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     if (lane == 0) {
       uint32_t it = 0;                       // k-block counter across tiles: the ring never restarts
       bool ok = true;
+      const uint64_t keep = l2_policy_evict_last();        // B is a weight matrix in every use of this kernel
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
         const int m0 = (tile / n_tiles) * BM, n0 = (tile % n_tiles) * BN;
         for (int kb = 0; kb < num_kb; ++kb, ++it) {
@@ -84,7 +85,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           if (!ok) break;
           mbar_expect_tx(&full[s], C::kABytes + C::kBBytes);
           tma_load_2d(sA + s * C::kABytes, &tmA, &full[s], kb * BK, m0);
-          tma_load_2d(sB + s * C::kBBytes, &tmB, &full[s], kb * BK, n0);
+          tma_load_2d_hint(sB + s * C::kBBytes, &tmB, &full[s], kb * BK, n0, keep);
         }
       }
     }
@@ -404,6 +405,7 @@ gemm_lstm_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
   if (!active) {
   } else if (warp == 0) {
     if (lane == 0) {
+      const uint64_t keep = l2_policy_evict_last();        // the gate weights: read again by every step
       for (int kb = 0; kb < num_kb; ++kb) {
         const int s = kb % kWideStages;
         const uint32_t ph = (kb / kWideStages) & 1;
@@ -412,8 +414,8 @@ gemm_lstm_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         tma_load_2d(sA + s * kWideABytes, &tmA, &full[s], kb * BK, m0);
         uint8_t* bdst = sB + s * kWideBBytes;
         int r = 0;
-        for (; r + 64 <= w; r += 64) tma_load_2d(bdst + r * (BK * 2), &tmB64, &full[s], kb * BK, n0 + r);
-        if (r < w) tma_load_2d(bdst + r * (BK * 2), &tmB32, &full[s], kb * BK, n0 + r);
+        for (; r + 64 <= w; r += 64) tma_load_2d_hint(bdst + r * (BK * 2), &tmB64, &full[s], kb * BK, n0 + r, keep);
+        if (r < w) tma_load_2d_hint(bdst + r * (BK * 2), &tmB32, &full[s], kb * BK, n0 + r, keep);
       }
     }
   } else if (warp == 1) {
