@@ -98,6 +98,7 @@ struct FusedJoinerParams {
   float* ldphi; float* la; float* lse;   // [R], [R][S], [R][S]
   float* ldnb;                       // [R][V] delta_nb as a probability ratio, NOT its log (0 at the blank column)
   int* err;
+  int* clear_word;                   // optional: one device word the kernel sets to 0 once its predecessors have finished
 };
 bool fused_joiner_eligible(int S, int V, int J);
 bool fused_joiner_specialised(int S);   // a kernel instance with this segment size compiled in exists

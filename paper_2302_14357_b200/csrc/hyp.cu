@@ -6,6 +6,8 @@
 // Scores are carried in float64: a hypothesis' log-probability reaches thousands of nats, where
 // float32 spacing (1.2e-4 at 2048) is coarser than the accuracy the stage kernels deliver.  The
 // stage kernels work on values relative to the row's score, which stay small.
+#include <cuda_bf16.h>
+
 #include "tw_internal.cuh"
 
 namespace tw {
@@ -100,7 +102,7 @@ __device__ __forceinline__ unsigned long long order_key(double x) {
 }
 
 __global__ void __launch_bounds__(2 * kStepThreads) hyp_step_kernel(HypState hs) {
-  __shared__ int s_nB, s_hasthr, s_nkeep;
+  __shared__ int s_nB, s_hasthr, s_nkeep, s_wbase;
   __shared__ int s_found[kMaxBeam], s_touched[kMaxBeam], s_carry[kMaxBeam];
   __shared__ double s_Als[kMaxBeam], s_Adone[kMaxBeam];
   __shared__ int s_Aslot[kMaxBeam], s_Alen[kMaxBeam];
@@ -385,6 +387,7 @@ __global__ void __launch_bounds__(2 * kStepThreads) hyp_step_kernel(HypState hs)
       if (passm != 0 && (capped || (passm & ~keepm) != 0)) hs.status[b] = TW_ERR_LIMIT;   // pass cap or token capacity
       s_nkeep = nk;
       hs.nA[b] = nk; hs.n_new[b] = nk;
+      s_wbase = (hs.inline_gather && nk > 0) ? atomicAdd(&hs.scalars[kScNPred], nk) : 0;   // this utterance's work-list entries
     }
   }
   __syncthreads();
@@ -410,6 +413,11 @@ __global__ void __launch_bounds__(2 * kStepThreads) hyp_step_kernel(HypState hs)
       hs.A_slot[b * kMaxBeam + i] = s_keep_slot[i];
       hs.A_ls[b * kMaxBeam + i] = s_keep_ls[i];
     }
+    if (hs.inline_gather && lane == 0) {           // the predictor's work-list entry of this hypothesis
+      const int wrow = s_wbase + i;
+      if (wrow < hs.B * hs.N) { hs.pw_new[wrow] = (int)gn; hs.pw_par[wrow] = (int)gp; hs.pw_tok[wrow] = k; }
+      else hs.status[b] = TW_ERR_LIMIT;            // cannot happen: the list holds at most N entries per utterance
+    }
     const long long r = r0 + h;
     // d_h(k) at frame t of the segment: occupancy times J(t, k)
     auto d_at = [&](int t) -> double {
@@ -429,6 +437,33 @@ __global__ void __launch_bounds__(2 * kStepThreads) hyp_step_kernel(HypState hs)
       // emitted at frame t: the hypothesis continues at frame t + 1, or has left the segment
       for (int t = lane; t < S; t += 32) hs.A_ld[((long long)b * kMaxBeam + i) * S + t] = t < slen ? d_at(t - 1) : -INFINITY;
       if (lane == 0) hs.A_done[b * kMaxBeam + i] = d_at(slen - 1);
+    }
+  }
+  // ---- the parents' h of every layer as bf16 in the recurrent halves of the gate GEMMs' operand rows (all threads:
+  // 16-byte pieces, independent of each other)
+  if (hs.inline_gather && nk > 0 && s_wbase + nk <= hs.B * hs.N) {
+    const long long stride = (long long)hs.L * 2 * hs.Hd;
+    const bool vec = (hs.Hd & 7) == 0 && (reinterpret_cast<uintptr_t>(hs.slot_hc) & 15) == 0;
+    const int per = vec ? hs.Hd >> 3 : hs.Hd;                 // pieces per (hypothesis, layer)
+    const int total = nk * hs.L * per;
+    for (int c = threadIdx.x; c < total; c += blockDim.x) {
+      const int i = c / (hs.L * per), rem = c - i * (hs.L * per), l = rem / per, x = rem - l * per;
+      const long long gp = bS + s_Aslot[s_keep_h[i]];
+      const float* hsrc = hs.slot_hc + gp * stride + (long long)l * 2 * hs.Hd;
+      __nv_bfloat16* d = reinterpret_cast<__nv_bfloat16*>(hs.xg_dst[l]) + (long long)(s_wbase + i) * hs.xg_ld[l] + hs.xg_off[l];
+      if (vec && (reinterpret_cast<uintptr_t>(d) & 15) == 0) {
+        const float4 a = *reinterpret_cast<const float4*>(hsrc + x * 8), e = *reinterpret_cast<const float4*>(hsrc + x * 8 + 4);
+        __nv_bfloat162 p0 = __floats2bfloat162_rn(a.x, a.y), p1 = __floats2bfloat162_rn(a.z, a.w);
+        __nv_bfloat162 p2 = __floats2bfloat162_rn(e.x, e.y), p3 = __floats2bfloat162_rn(e.z, e.w);
+        uint4 pk;
+        pk.x = *reinterpret_cast<uint32_t*>(&p0); pk.y = *reinterpret_cast<uint32_t*>(&p1);
+        pk.z = *reinterpret_cast<uint32_t*>(&p2); pk.w = *reinterpret_cast<uint32_t*>(&p3);
+        *reinterpret_cast<uint4*>(d + x * 8) = pk;
+      } else if (vec) {
+        for (int u = 0; u < 8; ++u) d[x * 8 + u] = __float2bfloat16_rn(hsrc[x * 8 + u]);
+      } else {
+        d[x] = __float2bfloat16_rn(hsrc[x]);
+      }
     }
   }
   // ---- list A empty: this segment is done ------------------------------------------------------

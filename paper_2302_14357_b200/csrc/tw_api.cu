@@ -1,4 +1,5 @@
 // C ABI of libtw: handle life-cycle, the decode driver and the separately callable stages.
+#include <stdlib.h>
 #include <new>
 #include <vector>
 #include <stdio.h>
@@ -68,7 +69,7 @@ void gemm_bf16(tw_handle* h, const Bf16Mat& A, const Bf16Mat& B, const int* M_de
 // output W_p g goes to row (idx_out ? idx_out[i] : i) of Pp_out.  State rows are [L][2][Hd].
 void enqueue_predictor(tw_handle* h, const int* tok, const float* hc_in, const int* idx_in, float* hc_out,
                        const int* idx_out, float* Pp_out, const int* n_dev, int n_max, cudaStream_t st,
-                       int* launches, const WorkListBuild* wl = nullptr) {
+                       int* launches, const WorkListBuild* wl = nullptr, bool gathered = false) {
   GemmOperand none{};
   if (h->pred_kind == TW_PRED_STATELESS) {
     GemmOperand a{h->emb, tok, h->emb_dim, h->W_p, h->P, h->P};
@@ -85,7 +86,7 @@ void enqueue_predictor(tw_handle* h, const int* tok, const float* hc_in, const i
     g.hc = hc_in; g.idx = idx_in; g.stride = stride; g.L = L; g.Hd = Hd;
     for (int l = 0; l < L; ++l) { g.dst[l] = h->bf.X[l].ptr; g.ld[l] = (int)h->bf.X[l].K; g.off[l] = (l == 0) ? 0 : Hd; }
     if (wl) g.wl = *wl;                       // the gather kernel builds tok / idx_in / idx_out / *n_dev first
-    launch_gather_parents_bf16(g, n_dev, n_max, st);
+    if (!gathered) launch_gather_parents_bf16(g, n_dev, n_max, st);   // gathered: hyp_step_kernel did both already
     // gate GEMMs with the LSTM cell in the epilogue; each writes the next GEMM's input half as bf16
     for (int l = 0; l < L; ++l) {
       GemmBf16Params p{n_dev, n_max, 4 * Hd, (int)h->bf.X[l].K, nullptr, nullptr, 0, nullptr, h->bf.err};
@@ -98,7 +99,7 @@ void enqueue_predictor(tw_handle* h, const int* tok, const float* hc_in, const i
         launch_gemm_bf16(h->bf.X[l].as_A, h->bf.W_cat[l].as_B128, h->bf.W_cat[l].as_B256, p, st);
     }
     gemm_bf16(h, h->bf.Htop, h->bf.W_p, n_dev, n_max, Pp_out, idx_out, h->J, nullptr, st);
-    *launches += L + 2;
+    *launches += L + (gathered ? 1 : 2);
     return;
   }
   for (int l = 0; l < L; ++l) {
@@ -139,8 +140,9 @@ void enqueue_predictor_slots(tw_handle* h, cudaStream_t st, int* launches, bool 
     wl.B = B; wl.n_new = hs.n_new; wl.new_slot = hs.new_slot; wl.new_par = hs.new_par; wl.new_tok = hs.new_tok;
     wl.pw_new = hs.pw_new; wl.pw_par = hs.pw_par; wl.pw_tok = hs.pw_tok; wl.n_out = hs.scalars + kScNPred;
   }
+  const bool gathered = build_list && h->hs_fused.inline_gather != 0;
   enqueue_predictor(h, hs.pw_tok, hs.slot_hc, hs.pw_par, hs.slot_hc, hs.pw_new, hs.slot_Pp,
-                    hs.scalars + kScNPred, h->R_max, st, launches, build_list ? &wl : nullptr);
+                    hs.scalars + kScNPred, h->R_max, st, launches, build_list && !gathered ? &wl : nullptr, gathered);
 }
 
 // E = enc W_e^T for `rows` frames
@@ -238,6 +240,7 @@ int build_bf16(tw_handle* h) {
     }
   }
   h->hs.defer_rows = 0;
+  h->hs.inline_gather = 0;
   h->hs.dnb_sel = nullptr;
   h->hs_fused = h->hs;
   h->hs_fused.logp = nullptr; h->hs_fused.lse = nullptr; h->hs_fused.ldphi_d = nullptr; h->hs_fused.la_d = nullptr;
@@ -249,6 +252,14 @@ int build_bf16(tw_handle* h) {
     h->hs_fused.defer_rows = h->aux_ok ? 1 : 0;
     h->hs_fused.dnb_sel = h->bf.ldnb_pad;        // the step's hyp_step_kernel picks the rows' best tokens itself
     h->hs_fused.V = h->bf.Vp;                    // row pitch of delta_nb there (padding columns hold 0)
+    // hyp_step_kernel builds the predictor's work list and operand rows itself (HypState::inline_gather)
+    const char* ig = getenv("TW_INLINE_GATHER");
+    if (h->hs_fused.defer_rows && h->pred_kind != TW_PRED_STATELESS && !(ig && ig[0] == '0')) {
+      h->hs_fused.inline_gather = 1;
+      for (int l = 0; l < h->L; ++l) {
+        h->hs_fused.xg_dst[l] = h->bf.X[l].ptr; h->hs_fused.xg_ld[l] = (int)h->bf.X[l].K; h->hs_fused.xg_off[l] = (l == 0) ? 0 : h->Hd;
+      }
+    }
   }
   TW_CUDA(h, cudaGetLastError());
   return TW_OK;
@@ -403,7 +414,7 @@ void enqueue_scan(tw_handle* h, const JoinerRows& rows, const float* ld_old, flo
 // Fused path: joiner, softmax, Eq. 3-7 and per-row candidates with the logits kept in tensor memory
 int enqueue_joiner_fused(tw_handle* h, const JoinerRows& rows, const float* ld_old, float* ldphi, float* ldnb,
                          float* la, const CandOut& cand, cudaStream_t st, int* launches, StageMarkFn mark_fn,
-                         bool plain_first, int utt_B) {
+                         bool plain_first, int utt_B, int* clear_word) {
   {
     PdlScope first(plain_first ? false : g_pdl_on);
     if (utt_B > 0) launch_joiner_A_tiled_utt(rows, h->hs.row_off, h->hs.nA, utt_B, h->bf.A_tiled.ptr, st);
@@ -414,7 +425,7 @@ int enqueue_joiner_fused(tw_handle* h, const JoinerRows& rows, const float* ld_o
   FusedJoinerParams fp{};
   fp.R_dev = rows.R_dev; fp.R_max = rows.R_max; fp.S = rows.S; fp.V = h->bf.Vp; fp.K = rows.J; fp.blank = h->blank;
   fp.CL = h->bf.CL; fp.no_max = h->bf.no_max ? 1 : 0; fp.bias = h->bf.bias_pad; fp.ld_old = ld_old; fp.row_slen = rows.row_slen;
-  fp.ldphi = ldphi; fp.la = la; fp.lse = h->bf.lse; fp.ldnb = ldnb; fp.err = h->bf.err;
+  fp.ldphi = ldphi; fp.la = la; fp.lse = h->bf.lse; fp.ldnb = ldnb; fp.err = h->bf.err; fp.clear_word = clear_word;
   TW_TRY(launch_fused_joiner(h->bf.A_tiled.as_A, h->bf.W_out_pad.as_B256, fp, h->bf.max_clusters, st));
   if (mark_fn) mark_fn(h, 2, st);       // the fused kernel alone
   *launches += 2;

@@ -112,7 +112,8 @@ typedef void (*StageMarkFn)(tw_handle*, int, cudaStream_t);
 int enqueue_joiner_fused(tw_handle* h, const JoinerRows& rows, const float* ld_old, float* ldphi, float* ldnb,
                          float* la, const CandOut& cand, cudaStream_t st, int* launches, StageMarkFn mark_fn = nullptr,
                          bool plain_first = false,    // plain_first: the operand kernel is launched with plain stream ordering
-                         int utt_B = 0);              // utt_B > 0: the rows are a decode step's (hs.row_off, hs.nA of utt_B utterances)
+                         int utt_B = 0,               // utt_B > 0: the rows are a decode step's (hs.row_off, hs.nA of utt_B utterances)
+                         int* clear_word = nullptr);  // a device word the fused kernel clears (FusedJoinerParams::clear_word)
 void enqueue_scan(tw_handle* h, const JoinerRows& rows, const float* ld_old, float* logp, float* ldphi,
                   float* ldnb, float* la, double* ldphi_d, double* la_d, const CandOut& cand, cudaStream_t st,
                   int* launches);

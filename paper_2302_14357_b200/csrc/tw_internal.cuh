@@ -179,6 +179,14 @@ struct HypState {
   float* cand_v; int* cand_k; int* cand_n;   // per-row expansion candidates [R][kMaxBeam], [R]
   // InitPredictor result (LSTM only): [L][2][Hd], [J]
   const float* init_hc; const float* init_Pp;
+  // inline_gather != 0 (fused bf16 decode with an LSTM predictor): hyp_step_kernel appends its new hypotheses to
+  // the predictor's work list itself (entries claimed by an atomic add on scalars[kScNPred], which the joiner
+  // kernel of the same pass cleared after the predictor kernels had read it) and writes their parents' h as bf16
+  // into the gate GEMMs' operand rows xg_dst[l] (row pitch xg_ld[l], column offset xg_off[l], in elements), so
+  // that no gather kernel runs between it and the first gate GEMM.  The order of the list's entries varies
+  // from run to run; no result depends on it (every entry is computed on its own).
+  int inline_gather;
+  void* xg_dst[kMaxLayers]; int xg_ld[kMaxLayers]; int xg_off[kMaxLayers];
 };
 
 void launch_hyp_init(const HypState& hs, const int* lengths, int B, int T, cudaStream_t st);
