@@ -324,3 +324,32 @@ np.savez(sys.argv[1], out=out.cpu().numpy(), Pp=Pp.cpu().numpy())
     assert np.all(np.isfinite(res["pair"]["out"]))
     np.testing.assert_allclose(res["pair"]["out"], res["single"]["out"], rtol=0, atol=1e-5)
     np.testing.assert_allclose(res["pair"]["Pp"], res["single"]["Pp"], rtol=0, atol=1e-4)
+
+
+def test_work_list_built_by_hyp_step_equals_gather_kernel(monkeypatch):
+    """Fused bf16 decode: the predictor's work list and operand rows written by hyp_step_kernel (entries in an
+    order that varies between runs) give the same decode, bit for bit, as the gather kernel's deterministic
+    list (TW_INLINE_GATHER=0, read by tw_init).  A ragged batch with a 2-layer LSTM, in both search variants."""
+    from paper_2302_14357_b200.binding import MODE_BF16, TwDecoder, weights_from_synth
+    cfg = tw_synth.WorkloadConfig("ig", 24, 60, (20, 60), 64, "lstm", 64, 2, 128, 128, 512, 3.0, 5, (3,), "bf16", 17)
+    m = tw_synth.make_model(cfg)
+    enc, lens = tw_synth.make_encoder_batch(cfg)
+    runs = {}
+    for flag in ("1", "0"):
+        monkeypatch.setenv("TW_INLINE_GATHER", flag)
+        dec = TwDecoder(weights_from_synth(m), N=cfg.N, S=3, mode=MODE_BF16, max_batch=cfg.batch, max_T=cfg.T)
+        out = []
+        for mono in (False, True):
+            dec.set_monotonic(mono)
+            out.append([x.cpu().numpy() for x in dec.decode(enc, lens)[:4]])
+            out.append(dec.stats())
+        dec.close()
+        runs[flag] = out
+    for a, b in zip(runs["1"], runs["0"]):
+        if isinstance(a, dict):
+            for key in ("frames", "calls", "joins", "rows", "limit_hits"):
+                assert a[key] == b[key], key
+            assert a["kernel_launches"] < b["kernel_launches"]          # one kernel fewer per step
+        else:
+            for x, y in zip(a, b):
+                np.testing.assert_array_equal(x, y)
