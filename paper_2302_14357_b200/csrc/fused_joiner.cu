@@ -35,6 +35,9 @@ constexpr int kColGroups = 4;                // epilogue warps per TMEM lane qua
 constexpr int kEpiWarps = 4 * kColGroups, kEpiThreads = 32 * kEpiWarps;
 constexpr int kThreadsFused = 64 + kEpiThreads;
 constexpr uint32_t kABytes = BM * BK * 2, kBBytes = NC * BK * 2;
+// long segments (S = 8, 10): the sum over a hypothesis's frames goes through a per-warp staging tile in shared
+// memory, 16 columns at a time (row = TMEM lane, odd pitch: conflict-free row-per-lane writes)
+constexpr int kStagePitch = 17;
 
 struct FusedSmem {
   // offsets from the 1024-aligned base
@@ -46,7 +49,8 @@ struct FusedSmem {
   static constexpr size_t kZb = kPart + (size_t)kColGroups * BM * 8;                       // float  [BM]
   static constexpr size_t kBias = kZb + (size_t)BM * 4;                           // float  [NC]
   static constexpr size_t kBars = kBias + (size_t)NC * 4;                         // uint64 [16]
-  static constexpr size_t kTotal = kBars + 16 * 8 + 16;
+  static constexpr size_t kStage = kBars + 16 * 8 + 16;                           // float  [kEpiWarps][32][kStagePitch]
+  static constexpr size_t kTotal = kStage + (size_t)kEpiWarps * 32 * kStagePitch * 4;
 };
 constexpr size_t kSmemFused = FusedSmem::kTotal + 1024;
 
