@@ -48,8 +48,8 @@ def parse_args():
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures
 # summarised under profiles/ (same workload, same kernel); absent entries report null
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    # profiles/fused_joiner_kernel_c3.md: 16.868 MB read + 7 KB written per launch (mean of three)
-    ("c3", 3, "fused_joiner_kernel (contraction + softmax + Eq. 3-7, tcgen05, cluster of V/256 CTAs)"): 16875093,
+    # profiles/fused_joiner_kernel_c3.md: 16.869 MB read + 11 KB written per launch (mean of three)
+    ("c3", 3, "fused_joiner_kernel (contraction + softmax + Eq. 3-7, tcgen05, cluster of V/256 CTAs)"): 16879616,
 }
 
 
