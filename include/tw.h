@@ -115,7 +115,11 @@ typedef struct {
  * the workspace for max_batch utterances of up to max_T frames.  Synchronises the device.
  * Errors: TW_ERR_ARG for null pointers, N not in [1, TW_MAX_BEAM], S not in [1, TW_MAX_SEGMENT],
  * V - 1 < N (fewer non-blank tokens than the beam), blank outside [0, V), P inconsistent with the
- * predictor; TW_ERR_ALLOC / TW_ERR_CUDA otherwise.  *out is NULL on failure. */
+ * predictor; TW_ERR_ALLOC / TW_ERR_CUDA otherwise.  *out is NULL on failure.
+ * Environment variables (diagnostic switches between kernels that compute the same thing; bf16 mode):
+ *   TW_INLINE_GATHER=0  read by tw_init: the predictor's work list and operand rows of a decode step are built by
+ *                       a kernel of their own instead of inside the hypothesis-step kernel
+ *   TW_GEMM_PAIRS=1     read once per process: the LSTM gate GEMMs run on CTA pairs (tcgen05 cta_group::2) */
 int tw_init(const tw_model* host_model, const tw_config* host_cfg, tw_handle** out);
 int tw_destroy(tw_handle* h);
 
