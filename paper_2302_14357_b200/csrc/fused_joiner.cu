@@ -35,7 +35,7 @@ constexpr int kColGroups = 4;                // epilogue warps per TMEM lane qua
 constexpr int kEpiWarps = 4 * kColGroups, kEpiThreads = 32 * kEpiWarps;
 constexpr int kThreadsFused = 64 + kEpiThreads;
 constexpr uint32_t kABytes = BM * BK * 2, kBBytes = NC * BK * 2;
-// long segments (S = 8, 10): the sum over a hypothesis's frames goes through a per-warp staging tile in shared
+// longer segments (S = 5, 8, 10): the sum over a hypothesis's frames goes through a per-warp staging tile in shared
 // memory, 16 columns at a time (row = TMEM lane, odd pitch: conflict-free row-per-lane writes)
 constexpr int kStagePitch = 17;
 
