@@ -42,15 +42,35 @@ def parse_args():
     ap.add_argument("--no-fused", action="store_true", help="bf16 mode: staged joiner kernels instead of the fused one")
     ap.add_argument("--monotonic", action="store_true", help="the monotonic RNN-T variant (every output consumes a frame)")
     ap.add_argument("--cpu-frames", type=int, default=0, help="frames of the CPU-baseline sample (0: auto)")
+    ap.add_argument("--no-largest", action="store_true", help="skip the fused kernel's leg at the largest step shape")
+    ap.add_argument("--agreement-utterances", type=int, default=4, help="utterances of the bf16 top-1 agreement check (0: skip)")
     return ap.parse_args()
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures
-# summarised under profiles/ (same workload, same kernel); absent entries report null
+# DRAM traffic of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum per launch) from ncu captures
+# of this same kernel: "cold" is the first launches of a process, "warm" a launch inside a running decode.  Each
+# entry carries the digest of the kernel's sources at the time of the capture; once the sources differ the
+# counters no longer describe the kernel that runs and the bench reports null.
+KERNEL_SOURCES = ("fused_joiner.cu", "fused_joiner_kernel.inc", "fused_joiner_host.inc", "sm100.cuh")
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    # profiles/fused_joiner_kernel_c3.md: 16.869 MB read + 11 KB written per launch (mean of three)
-    ("c3", 3, "fused_joiner_kernel (contraction + softmax + Eq. 3-7, tcgen05, cluster of V/256 CTAs)"): 16879616,
+    # (workload, S): (source digest, cold bytes, warm bytes)
 }
+
+
+def kernel_source_digest():
+    import hashlib
+    h = hashlib.sha1()
+    for name in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_2302_14357_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:12]
+
+
+def ncu_traffic(workload, S):
+    ent = NCU_DRAM_BYTES_PER_LAUNCH.get((workload, S))
+    if ent is None or ent[0] != kernel_source_digest():
+        return None, None
+    return {"cold": ent[1], "warm": ent[2]}, ent[0]
 
 
 def joiner_kernel_name(mode_name, st):
@@ -97,6 +117,69 @@ def oracle_sample(cfg, S, frames, utt=0, monotonic=False):
             "sample": "utterance %d of workload %s, first %d frames, N=%d S=%d, fp64 numpy; %.1f s"
                       % (utt, cfg.name, n, cfg.N, S, dt),
             "calls_per_frame": st.calls / max(n, 1), "joins_per_frame": st.joins / max(n, 1)}, dt
+
+
+def top1_agreement(dec, cfg, S, enc_np, len_np, utterances, frames, monotonic=False):
+    """bf16 mode against the fp64 oracle: both decode the first `frames` frames of a few utterances of the
+    bench batch; reports how often the best token sequence is the same and the largest score gap where it is."""
+    from oracle import rnnt_model as rm
+    from oracle import token_wise_search as tws
+    K = int(min(utterances, enc_np.shape[0]))
+    F = int(min(frames, enc_np.shape[1]))
+    enc = np.ascontiguousarray(enc_np[:K, :F])
+    lens = np.minimum(len_np[:K], F).astype(np.int32)
+    tokens, olens, scores, status, _ = dec.decode(enc, lens)
+    tokens, olens, scores = tokens.cpu().numpy(), olens.cpu().numpy(), scores.cpu().numpy()
+    m = tw_synth.make_model(cfg)
+    om = rm.RnntModel(m.W_e, m.W_p, m.W_out, m.b_out, m.emb, m.lstm_W_ih, m.lstm_W_hh, m.lstm_b,
+                      activation=cfg.joiner_act)
+    agree, gap = 0, 0.0
+    for b in range(K):
+        ref, _ = tws.token_wise_beam_search(om, enc[b, :lens[b]], cfg.N, S, max_iters=4 * S + 16, monotonic=monotonic)
+        got = tuple(int(x) for x in tokens[b, 0, :max(int(olens[b, 0]), 0)])
+        if got == ref[0][0]:
+            agree += 1
+            gap = max(gap, abs(float(scores[b, 0]) - ref[0][1]))
+    return {"rate": agree / max(K, 1), "utterances": K, "frames_each": F, "max_score_gap": gap,
+            "against": "fp64 oracle on the same bf16-rounded weights and frames"}
+
+
+def largest_step_roofline(peaks, launches=20, warm=5):
+    """The fused joiner kernel alone at the largest step shape of the workloads: B = 512 utterances x N = 10
+    hypotheses x S = 10 frames = 51,200 joiner rows, V = 4096, J = 1024 (workload c4's model), timed with CUDA
+    events around the kernel (tw_set_profiling) through tw_joiner_expand.  Operand (105 MB) and delta_nb (84 MB)
+    exceed L2."""
+    import torch
+    from paper_2302_14357_b200.binding import MODE_BF16, TwDecoder, weights_from_synth
+    cfg = tw_synth.get_config("c4")
+    S, N, B = 10, cfg.N, cfg.batch
+    R = B * N
+    dec = TwDecoder(weights_from_synth(tw_synth.make_model(cfg)), N=N, S=S, mode=MODE_BF16, max_batch=B, max_T=2 * S)
+    if not dec.set_fused(True):
+        return None
+    g = torch.Generator(device="cuda").manual_seed(4)
+    E = torch.randn((B, S, cfg.J), device="cuda", generator=g)
+    Pp = torch.randn((R, cfg.J), device="cuda", generator=g) * 0.5
+    row_group = (torch.arange(R, device="cuda", dtype=torch.int32) // N).contiguous()
+    ld_old = torch.randn((R, S), device="cuda", generator=g) - 2.0
+    for _ in range(warm):
+        dec.joiner_expand(E, Pp, row_group, None, ld_old)
+    dec.set_profiling(True)
+    for _ in range(launches):
+        dec.joiner_expand(E, Pp, row_group, None, ld_old)
+    st = dec.stats()
+    dec.set_profiling(False)
+    dec.close()
+    if st["joiner_launches"] <= 0 or st["ns_joiner"] <= 0:
+        return None
+    us = st["ns_joiner"] * 1e-3 / st["joiner_launches"]
+    flops = 2.0 * cfg.J * cfg.V * R * S
+    achieved = flops / (us * 1e-6) / 1e12
+    return {"workload": "c4-step (R=%d rows x S=%d frames, V=%d, J=%d)" % (R, S, cfg.V, cfg.J),
+            "kernel": "fused_joiner_kernel", "bound": "tensor", "achieved": achieved, "unit": "TFLOP/s",
+            "peak": peaks["tflops_sustained"], "frac": achieved / peaks["tflops_sustained"],
+            "frac_burst": achieved / peaks["tflops_burst"], "avg_launch_us": us, "launches": int(st["joiner_launches"]),
+            "flops_per_launch": flops, "operand_kernel_avg_us": st["ns_scan"] * 1e-3 / st["joiner_launches"]}
 
 
 def auto_cpu_frames(cfg):
@@ -280,6 +363,23 @@ def run_ours(args, cfg, S):
     peak = peaks["tflops_sustained"]
     stage_ns = {k: st[k] for k in ("ns_prologue", "ns_predictor", "ns_joiner", "ns_scan", "ns_hyp")}
     tot_ns = max(1, sum(stage_ns.values()))
+    traffic, traffic_rev = ncu_traffic(cfg.name, S) if (mode_name == "bf16" and st.get("fused_on")) else (None, None)
+    # the HBM-side kernels of a step, from the same stage events: algorithmic bytes per decode / device time
+    fused = mode_name == "bf16" and st.get("fused_on")
+    hbm = {}
+    if fused and st["steps"] > 0:
+        rows, frame_rows, steps = st["rows"], st["joiner_frame_rows"], st["steps"]
+        # hyp_step_kernel: every row's delta_nb [V] float32 read once (selection) + per row about 64 B of list state
+        b_hyp = rows * (4.0 * dec.Vp + 64.0)
+        # operand kernel: E rows (float32) and Pp rows (float32) read, act(E + Pp) written as bf16
+        b_op = frame_rows * cfg.J * (4.0 + 2.0) + rows * cfg.J * 4.0
+        for name, nbytes, ns in (("hyp_step_kernel (selection over delta_nb, AddAndMerge, threshold, new list A)", b_hyp, st["ns_hyp"]),
+                                 ("joiner_A_tiled_kernel (operand act(E + Pp) as bf16)", b_op, st["ns_scan"])):
+            if ns > 0:
+                gbs = nbytes / (ns * 1e-9) / 1e9
+                hbm[name.split(" ")[0]] = {"kernel": name, "bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                           "frac": gbs / peaks["hbm_gbs"], "avg_launch_us": ns * 1e-3 / steps,
+                                           "bytes_per_launch": nbytes / steps}
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms / args.steps, "ms_per_step_with_stage_events": ms_profiled / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -294,8 +394,12 @@ def run_ours(args, cfg, S):
         "stage_share": {k[3:]: round(v / tot_ns, 4) for k, v in stage_ns.items()},
         "stage_ms_per_decode": {k[3:]: round(v * 1e-6, 3) for k, v in stage_ns.items()},
         "roofline": {"kernel": joiner_kernel_name(mode_name, st), "bound": "tensor", "achieved": achieved, "peak": peak,
-                     "unit": "TFLOP/s", "frac": achieved / peak if peak else None, "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get((cfg.name, S, joiner_kernel_name(mode_name, st))),
-                     "peak_source": "%s bf16 sustained" % peaks["source"],
+                     "unit": "TFLOP/s", "frac": achieved / peak if peak else None,
+                     "frac_sustained": achieved / peaks["tflops_sustained"], "frac_burst": achieved / peaks["tflops_burst"],
+                     "peak_burst": peaks["tflops_burst"],
+                     "traffic": traffic, "traffic_kernel_digest": traffic_rev,
+                     "peak_source": "%s bf16 sustained (a seconds-long cuBLAS loop under the power cap); frac_burst is against the "
+                                    "burst figure, measured at the SM clock in `clocks`" % peaks["source"],
                      "avg_launch_us": 1e6 * joiner_s / max(st["joiner_launches"], 1),
                      "flops_per_launch": st["joiner_frame_rows"] * flops_per_row / max(st["joiner_launches"], 1)},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(enc_np.nbytes + len_np.nbytes),
@@ -303,6 +407,15 @@ def run_ours(args, cfg, S):
         "gpu_launches": int(st["kernel_launches"] * args.steps),
         "clocks": clocks,
     }
+    if hbm:
+        line["roofline_hbm"] = hbm
+    if mode_name == "bf16" and world == 1 and not args.no_largest:
+        big = largest_step_roofline(peaks)
+        if big is not None:
+            line["roofline_largest"] = big
+    if mode_name == "bf16" and world == 1 and not args.no_cpu_baseline and args.agreement_utterances > 0:
+        line["bf16_top1_agreement"] = top1_agreement(dec, cfg, S, enc_np, len_np, args.agreement_utterances,
+                                                     min(150, args.cpu_frames or auto_cpu_frames(cfg)), args.monotonic)
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"], _ = oracle_sample(cfg, S, args.cpu_frames or auto_cpu_frames(cfg), monotonic=args.monotonic)
     print(json.dumps(line))

@@ -52,7 +52,7 @@ enum { TW_ACT_TANH = 0, TW_ACT_RELU = 1 };   /* joiner hidden nonlinearity */
 /*
  * The RNN-T pieces the search calls (Sec. 3.1).
  *   joiner:    z(t,u,.) = W_out . act(W_e h_t + W_p g_u) + b_out,  J = softmax(z); act = tanh, or ReLU
- *              (the paper's models use "a ReLU layer followed by a single fully connected layer", Sec. 4.1)
+ *              (TW_ACT_RELU is the joiner of the models in Sec. 4.1)
  *   predictor: stateless  g = emb[last token]         (P == emb_dim; empty prefix -> emb[blank])
  *              LSTM       lstm_layers stacked cells, gate order (input, forget, cell, output),
  *                         one bias per layer, g = top layer's h   (P == lstm_hidden);
@@ -115,11 +115,8 @@ typedef struct {
  * the workspace for max_batch utterances of up to max_T frames.  Synchronises the device.
  * Errors: TW_ERR_ARG for null pointers, N not in [1, TW_MAX_BEAM], S not in [1, TW_MAX_SEGMENT],
  * V - 1 < N (fewer non-blank tokens than the beam), blank outside [0, V), P inconsistent with the
- * predictor; TW_ERR_ALLOC / TW_ERR_CUDA otherwise.  *out is NULL on failure.
- * Environment variables (diagnostic switches between kernels that compute the same thing; bf16 mode):
- *   TW_INLINE_GATHER=0  read by tw_init: the predictor's work list and operand rows of a decode step are built by
- *                       a kernel of their own instead of inside the hypothesis-step kernel
- *   TW_GEMM_PAIRS=1     read once per process: the LSTM gate GEMMs run on CTA pairs (tcgen05 cta_group::2) */
+ * predictor; TW_ERR_ALLOC / TW_ERR_CUDA otherwise.  *out is NULL on failure.  The library reads no environment
+ * variable: every switch is a call on the handle. */
 int tw_init(const tw_model* host_model, const tw_config* host_cfg, tw_handle** out);
 int tw_destroy(tw_handle* h);
 
@@ -250,6 +247,8 @@ int tw_predictor_step(tw_handle* h, const int32_t* tokens, const float* state_in
  * process exits).  The call itself never calls cudaMalloc, cudaFree or any allocating routine.
  *
  *   W_out [V, J], b_out [V]   joiner output layer (float32, device)
+ *   joiner_act                TW_ACT_TANH or TW_ACT_RELU: the joiner's hidden nonlinearity (a handle carries it in
+ *                             its model; here it has to be said)
  *   the remaining arguments are those of tw_joiner_expand, computed in float32
  * Limits: R <= TW_NOALLOC_MAX_ROWS and R * S * V <= TW_NOALLOC_MAX_ELEMS; a larger request returns
  * TW_ERR_LIMIT and enqueues nothing.  Other bad arguments return TW_ERR_ARG.
@@ -263,7 +262,7 @@ int tw_predictor_step(tw_handle* h, const int32_t* tokens, const float* state_in
 #define TW_NOALLOC_MAX_ROWS 4096
 #define TW_NOALLOC_MAX_ELEMS (4 * 1024 * 1024)
 int tw_joiner_expand_noalloc(const float* W_out, const float* b_out, int32_t J, int32_t V, int32_t S,
-                             int32_t blank, const float* E_seg, const float* Pp,
+                             int32_t blank, int32_t joiner_act, const float* E_seg, const float* Pp,
                              const int32_t* row_group, const int32_t* seg_len, const float* ld_old,
                              int32_t G, int32_t R, float* out_ldphi, float* out_ldnb, float* out_la,
                              void* stream);
@@ -272,8 +271,7 @@ int tw_joiner_expand_noalloc(const float* W_out, const float* b_out, int32_t J, 
  * kept in tensor memory; available when S <= 32 and V <= 4096, a vocabulary that is not a multiple of 256
  * being padded internally with columns of probability 0; the default for S in {1..5, 8, 10}) and the
  * staged kernels that pass the logits through device memory.  Both compute the same quantities.
- * tw_joiner_expand uses the fused kernel only with an unpadded vocabulary (its delta_nb rows have V
- * columns).  TW_ERR_STATE if the fused kernel is not available for this handle. */
+ * TW_ERR_STATE if the fused kernel is not available for this handle. */
 int tw_set_fused(tw_handle* h, int on);
 
 /* tw_decode replays its step body (16 device steps) as a CUDA graph, captured once per batch shape, on
@@ -287,6 +285,12 @@ int tw_set_graph(tw_handle* h, int on);
  * tw_set_lanes(h, 0) decodes the batch in one piece.  Default: on.  Off while profiling is on. */
 int tw_set_lanes(tw_handle* h, int on);
 
+/* TW_MODE_BF16 with the fused joiner and an LSTM predictor: by default the hypothesis-step kernel of a decode step also
+ * builds the predictor's work list and writes the parents' recurrent states into the gate GEMMs' operand rows;
+ * tw_set_inline_gather(h, 0) leaves both to a kernel of their own (one more launch per step, a work list in a fixed
+ * order).  Both give the same N-best.  TW_ERR_STATE if the handle has no such path, or while a streaming session is open. */
+int tw_set_inline_gather(tw_handle* h, int on);
+
 /* Monotonic RNN-T variant (Sec. 2 and Sec. 5 name it as an adjustment of Algorithm 1; the paper prints no
  * equations for it).  Every output, blank or token, consumes one frame, so at most one token is emitted
  * per frame.  In Eq. 4-5 a token emitted at frame t2 leaves its hypothesis at frame t2 + 1, and a
@@ -296,7 +300,10 @@ int tw_set_lanes(tw_handle* h, int on);
 int tw_set_monotonic(tw_handle* h, int on);
 
 /* Per-stage device timing of tw_decode with CUDA events on the decode stream (adds two event records
- * per stage per step); off by default. */
+ * per stage per step); off by default.  While it is on, tw_joiner_expand on the fused path also times its two
+ * kernels: each call synchronises `stream` and ADDS the operand kernel's device time to ns_scan, the fused
+ * kernel's to ns_joiner and 1 to joiner_launches (tw_get_stats).  Every call of tw_set_profiling clears those
+ * three counters. */
 int tw_set_profiling(tw_handle* h, int on);
 int tw_get_stats(const tw_handle* h, tw_stats* host_out);
 int tw_last_cuda_error(const tw_handle* h); /* cudaError_t of the last failed CUDA call, 0 if none */

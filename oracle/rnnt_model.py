@@ -2,7 +2,8 @@
 softmax normalisation J, and the prediction network g(u).  fp64 throughout.
 
 Joiner form: z = W_out . act(W_e h_t + W_p g_u) + b_out with act = tanh (the synthetic benchmark
-workloads) or ReLU (the paper's models: a ReLU layer followed by one fully connected layer, Sec. 4.1).
+workloads) or ReLU (the joiner of the models in Sec. 4.1: one rectified hidden layer, then a linear map to
+the vocabulary).
 Predictor: either stateless (g = embedding of the last token; the empty
 prefix uses the blank token's embedding) or a stack of LSTM layers with gate
 order (input, forget, cell, output) and a single bias per layer, started by
@@ -83,6 +84,24 @@ def lstm_step(model: RnntModel, state: PredState, token: int):
         c_new.append(c)
         x = h
     return (h_new, c_new), x
+
+
+def lstm_step_rows(model: RnntModel, h_prev: np.ndarray, c_prev: np.ndarray, tokens: Sequence[int]):
+    """The same predictor step as lstm_step for R hypotheses at once (UpdatePredictorOutput of Algorithm 1
+    runs the predictor for every new hypothesis; Sec. 4.1: a stack of LSTM layers).
+    h_prev, c_prev [R, L, Hd], tokens [R] -> (h_new [R, L, Hd], c_new [R, L, Hd], out [R, Hd])."""
+    h_prev, c_prev = _f64(h_prev), _f64(c_prev)
+    x = model.emb[np.asarray(tokens, dtype=np.int64)]            # [R, emb_dim]
+    h_new, c_new = np.empty_like(h_prev), np.empty_like(c_prev)
+    for l in range(len(model.lstm_W_ih)):
+        gates = x @ model.lstm_W_ih[l].T + h_prev[:, l] @ model.lstm_W_hh[l].T + model.lstm_b[l]
+        Hd = gates.shape[1] // 4
+        i, f, g, o = (gates[:, 0:Hd], gates[:, Hd:2 * Hd], gates[:, 2 * Hd:3 * Hd], gates[:, 3 * Hd:4 * Hd])
+        c = _sigmoid(f) * c_prev[:, l] + _sigmoid(i) * np.tanh(g)
+        h = _sigmoid(o) * np.tanh(c)
+        h_new[:, l], c_new[:, l] = h, c
+        x = h
+    return h_new, c_new, x
 
 
 def predictor_init(model: RnntModel):

@@ -1,5 +1,10 @@
 """Algorithm 1: token-wise beam search for RNN-T, one utterance, fp64 log space.
 
+`token_wise_beam_search` takes the steps of Algorithm 1 in the order the paper gives them and with its
+names (lists A and B, ChooseNBest, AddAndMerge, ChooseNthScore, ChooseNBestExpansions,
+UpdatePredictorOutput), so that it can be checked against the algorithm by eye; the code is written
+from the algorithm's description, with Eq. 3-7 taken from segment_math.
+
 Readings of points the paper leaves open (each mirrored by the CUDA path):
   * last segment when S does not divide the length: seg = enc[t:t+S] is a
     slice, so the final segment is simply shorter (S' = len - t);

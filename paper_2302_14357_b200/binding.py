@@ -12,7 +12,7 @@ TW_OK, TW_ERR_ARG, TW_ERR_ALLOC, TW_ERR_CUDA, TW_ERR_LIMIT, TW_ERR_STATE, TW_ERR
 
 EXPORTED_SYMBOLS = [
     "tw_init", "tw_destroy", "tw_decode", "tw_decode_host", "tw_max_tokens", "tw_project_encoder",
-    "tw_joiner_segment", "tw_expand", "tw_joiner_expand", "tw_predictor_step", "tw_get_stats", "tw_set_profiling", "tw_set_fused", "tw_set_graph", "tw_set_lanes", "tw_set_monotonic",
+    "tw_joiner_segment", "tw_expand", "tw_joiner_expand", "tw_predictor_step", "tw_get_stats", "tw_set_profiling", "tw_set_fused", "tw_set_graph", "tw_set_lanes", "tw_set_monotonic", "tw_set_inline_gather",
     "tw_stream_open", "tw_stream_push", "tw_stream_nbest", "tw_stream_close",
     "tw_joiner_expand_noalloc",
     "tw_last_cuda_error", "tw_strerror",
@@ -74,11 +74,12 @@ def load_library() -> C.CDLL:
     lib.tw_set_graph.argtypes = [vp, C.c_int]
     lib.tw_set_lanes.argtypes = [vp, C.c_int]
     lib.tw_set_monotonic.argtypes = [vp, C.c_int]
+    lib.tw_set_inline_gather.argtypes = [vp, C.c_int]
     lib.tw_stream_open.argtypes = [vp, i32, vp]
     lib.tw_stream_push.argtypes = [vp, vp, vp, i32, vp]
     lib.tw_stream_nbest.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.tw_stream_close.argtypes = [vp, vp, vp, vp, vp, vp]
-    lib.tw_joiner_expand_noalloc.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp]
+    lib.tw_joiner_expand_noalloc.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp]
     lib.tw_last_cuda_error.argtypes = [vp]
     lib.tw_strerror.argtypes = [C.c_int]
     lib.tw_strerror.restype = C.c_char_p
@@ -148,6 +149,7 @@ class TwDecoder:
         self.L, self.Hd = layers, m.lstm_hidden
         self.mode = mode
         self.U_cap = self.lib.tw_max_tokens(self.h)
+        self.Vp = (V + 255) // 256 * 256      # row pitch of delta_nb on the fused path (vocabulary padded to 256 columns)
 
     # -- helpers -------------------------------------------------------------------------------
     def _stream(self):
@@ -293,6 +295,10 @@ class TwDecoder:
         """tw_set_monotonic: the monotonic RNN-T variant (every output consumes a frame) for later decodes."""
         self._check(self.lib.tw_set_monotonic(self.h, int(bool(on))), "tw_set_monotonic")
 
+    def set_inline_gather(self, on: bool):
+        """tw_set_inline_gather: who builds the predictor's work list in a fused bf16 decode step."""
+        self._check(self.lib.tw_set_inline_gather(self.h, int(bool(on))), "tw_set_inline_gather")
+
     def set_lanes(self, on: bool):
         self._check(self.lib.tw_set_lanes(self.h, int(bool(on))), "tw_set_lanes")
 
@@ -316,7 +322,7 @@ NOALLOC_MAX_ROWS = 4096
 NOALLOC_MAX_ELEMS = 4 * 1024 * 1024
 
 
-def joiner_expand_noalloc(W_out, b_out, S, blank, E_seg, Pp, row_group, seg_len, ld_old):
+def joiner_expand_noalloc(W_out, b_out, S, blank, E_seg, Pp, row_group, seg_len, ld_old, joiner_act="tanh"):
     """tw_joiner_expand_noalloc: joiner + softmax + Eq. 3-7 without a handle and without any device
     allocation inside the library (its scratch is a fixed array in the library image).  All arguments
     are CUDA tensors the caller already owns (float32, int32 for row_group / seg_len); the three
@@ -329,7 +335,8 @@ def joiner_expand_noalloc(W_out, b_out, S, blank, E_seg, Pp, row_group, seg_len,
     ldphi = torch.empty((R,), dtype=torch.float32, device=dev)
     ldnb = torch.empty((R, V), dtype=torch.float32, device=dev)
     la = torch.empty((R, S), dtype=torch.float32, device=dev)
-    st = lib.tw_joiner_expand_noalloc(W_out.data_ptr(), b_out.data_ptr(), J, V, S, blank, E_seg.data_ptr(), Pp.data_ptr(),
+    act = joiner_act if isinstance(joiner_act, int) else {"tanh": ACT_TANH, "relu": ACT_RELU}[joiner_act]
+    st = lib.tw_joiner_expand_noalloc(W_out.data_ptr(), b_out.data_ptr(), J, V, S, blank, act, E_seg.data_ptr(), Pp.data_ptr(),
                                       row_group.data_ptr(), _ptr(seg_len), ld_old.data_ptr(), G, R, ldphi.data_ptr(),
                                       ldnb.data_ptr(), la.data_ptr(), torch.cuda.current_stream().cuda_stream)
     return st, ldphi, ldnb, la

@@ -47,7 +47,7 @@ void launch_gemm_bf16(const CUtensorMap& tmA, const CUtensorMap& tmB128, const C
 // nearly empty wave; returns false (nothing launched) when the shape does not call for it.
 // tmB64 / tmB32: maps of B with 64- and 32-row boxes
 bool launch_gemm_lstm_wide(const CUtensorMap& tmA, const CUtensorMap& tmB64, const CUtensorMap& tmB32,
-                           const GemmBf16Params& p, cudaStream_t st, const CUtensorMap* tmB16 = nullptr);
+                           const GemmBf16Params& p, cudaStream_t st);
 
 // A bf16 matrix with its tensor maps
 struct Bf16Mat {
@@ -55,7 +55,7 @@ struct Bf16Mat {
   long long rows = 0, K = 0;
   CUtensorMap as_A;            // box 128 rows
   CUtensorMap as_B128, as_B256;
-  CUtensorMap as_B64, as_B32, as_B16;
+  CUtensorMap as_B64, as_B32;
 };
 
 // elementwise helpers ---------------------------------------------------------------------------
@@ -106,8 +106,9 @@ long long fused_joiner_A_rows(int R_max, int S);      // rows of the tile-layout
 int fused_joiner_setup(int CL, int S, int* max_clusters);
 // max_k (sum_j |W_out[k, j]| + |b_out[k]|): bound of |z| since |tanh| <= 1; written to *out (device)
 void launch_logit_bound(const __nv_bfloat16* W, const float* bias, int V, int J, float* out, cudaStream_t st);
-// in place: x -> log x (log 0 = -inf), n elements
-void launch_log_inplace(float* x, long long n, cudaStream_t st);
+// dst[r, k] = log src[r * ld_src + k] (log 0 = -inf) for r < R, k < V; dst rows have V columns (dst may be src when
+// ld_src == V)
+void launch_log_rows(const float* src, long long ld_src, float* dst, int R, int V, cudaStream_t st);
 void launch_joiner_A_tiled(const JoinerRows& rows, __nv_bfloat16* A, cudaStream_t st);
 // the same for the rows of a decode step (utterance b's rows are row_off[b] .. + nA[b] - 1, all on one segment)
 void launch_joiner_A_tiled_utt(const JoinerRows& rows, const int* row_off, const int* nA, int B, __nv_bfloat16* A,

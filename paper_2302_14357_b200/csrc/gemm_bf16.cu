@@ -7,7 +7,6 @@
 // the kernel raises *err and every role leaves its loop.
 #include "bf16_path.cuh"
 #include "sm100.cuh"
-#include <stdlib.h>
 
 namespace tw {
 
@@ -449,121 +448,6 @@ gemm_lstm_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
   if (warp == 1) tmem_dealloc(tmem_base, 512);
 }
 
-// ---- the same GEMM on CTA pairs ------------------------------------------------------------------
-// The contraction above is bound by what an SM can pull from L2 (its A tile and its B slice per K step).  Here two
-// CTAs of a cluster share one MMA of M = 256 (tcgen05 cta_group::2): the pair owns 256 rows x w columns, each CTA
-// loads its 128 rows of A and HALF of the B slice, and gets its 128 rows of the accumulator in its own tensor
-// memory, so the epilogue is unchanged.  The even CTA issues the MMAs; both CTAs' loads are counted on its `full`
-// barriers; `empty` and `acc_full` arrivals are multicast to both.
-// a CTA of a pair holds at most half of a 320-column slice of B per stage: six stages fit where the single-CTA
-// kernel has four, which keeps the same number of bytes in flight per SM
-constexpr int kPairStages = 6;
-constexpr uint32_t kPairBBytes = (kWideMaxBN / 2) * BK * 2;
-constexpr size_t kPairSmem = (size_t)kPairStages * (kWideABytes + kPairBBytes) + 1024 + 256;
-__global__ void __launch_bounds__(kThreadsWide, 1)
-gemm_lstm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB64,
-                      const __grid_constant__ CUtensorMap tmB32, const __grid_constant__ CUtensorMap tmB16,
-                      GemmBf16Params p) {
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint8_t* sA = smem;
-  uint8_t* sB = smem + kPairStages * kWideABytes;
-  uint64_t* full = reinterpret_cast<uint64_t*>(sB + kPairStages * kPairBBytes);
-  uint64_t* empty = full + kPairStages;
-  uint64_t* acc_full = empty + kPairStages;
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(acc_full + 1);
-
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int num_kb = (p.K + BK - 1) / BK;
-  const uint32_t rank = cluster_ctarank();               // 0: issues the MMAs, 1: its peer
-
-  if (threadIdx.x == 0) {
-    prefetch_tensormap(&tmA);
-    prefetch_tensormap(&tmB64);
-    prefetch_tensormap(&tmB32);
-    prefetch_tensormap(&tmB16);
-    for (int s = 0; s < kPairStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    mbar_init(acc_full, 1);
-    fence_barrier_init();
-    fence_proxy_async_smem();
-  }
-  if (warp == 1) { tmem_alloc_pair(tmem_holder, 512); tmem_relinquish_pair(); }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_base = *tmem_holder;
-  cluster_sync_all();                                    // both CTAs' barriers exist before either signals the other
-  pdl_wait();
-  pdl_trigger();
-  const int M = p.M_dev ? *p.M_dev : p.M;
-  const int m_pairs = M > 0 ? (M + 2 * BM - 1) / (2 * BM) : 1;
-  const int units = p.N >> 5;
-  int n_split = (int)(gridDim.x >> 1) / m_pairs;
-  n_split = n_split < 1 ? 1 : (n_split > units ? units : n_split);
-  const int pair = blockIdx.x >> 1;
-  const int mp = pair / n_split, ns = pair - mp * n_split;
-  const int m0 = mp * 2 * BM + (int)rank * BM;           // this CTA's rows
-  const int ubase = units / n_split, urem = units - ubase * n_split;
-  const int u0 = ns * ubase + (ns < urem ? ns : urem), nu = ubase + (ns < urem ? 1 : 0);
-  const int n0 = u0 * 32, w = nu * 32;                   // the pair's columns [n0, n0 + w)
-  if (w > kWideMaxBN && threadIdx.x == 0) atomicExch(p.err, 1);
-  const bool active = mp < m_pairs && mp * 2 * BM < M && w > 0 && w <= kWideMaxBN;   // per pair: both CTAs agree
-  const int n1 = w < 256 ? w : 256, n2 = w - n1;         // two MMAs per K step when the slice is wider than 256
-  const int h1 = n1 >> 1, h2 = n2 >> 1;                  // B rows of each that THIS CTA holds
-
-  if (!active) {
-  } else if (warp == 0) {
-    if (lane == 0) {
-      const uint32_t stage_bytes = kWideABytes + (uint32_t)(h1 + h2) * (BK * 2);
-      for (int kb = 0; kb < num_kb; ++kb) {
-        const int s = kb % kPairStages;
-        const uint32_t ph = (kb / kPairStages) & 1;
-        if (!mbar_wait(&empty[s], ph ^ 1, p.err)) break;
-        if (rank == 0) mbar_expect_tx(&full[s], 2 * stage_bytes);          // this CTA's bytes and the peer's
-        const uint32_t bar = map_to_cta(smem_u32(&full[s]), 0);
-        tma_load_2d_pair(sA + s * kWideABytes, &tmA, bar, kb * BK, m0);
-        uint8_t* bdst = sB + s * kPairBBytes;
-        // rows [g, g + cnt) of B to shared-memory rows [d, d + cnt): boxes of 64, 32 and 16 rows
-        for (int part = 0; part < 2; ++part) {
-          int g = part == 0 ? n0 + (int)rank * h1 : n0 + n1 + (int)rank * h2;
-          int d = part == 0 ? 0 : h1, cnt = part == 0 ? h1 : h2;
-          for (; cnt >= 64; cnt -= 64, g += 64, d += 64) tma_load_2d_pair(bdst + d * (BK * 2), &tmB64, bar, kb * BK, g);
-          if (cnt >= 32) { tma_load_2d_pair(bdst + d * (BK * 2), &tmB32, bar, kb * BK, g); cnt -= 32; g += 32; d += 32; }
-          if (cnt >= 16) { tma_load_2d_pair(bdst + d * (BK * 2), &tmB16, bar, kb * BK, g); }
-        }
-      }
-    }
-  } else if (warp == 1) {
-    if (lane == 0 && rank == 0) {
-      const uint32_t idesc1 = make_idesc_bf16(2 * BM, n1), idesc2 = make_idesc_bf16(2 * BM, n2);
-      bool ok = true;
-      for (int kb = 0; kb < num_kb; ++kb) {
-        const int s = kb % kPairStages;
-        const uint32_t ph = (kb / kPairStages) & 1;
-        ok = mbar_wait(&full[s], ph, p.err);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t a_addr = smem_u32(sA + s * kWideABytes), b_addr = smem_u32(sB + s * kPairBBytes);
-#pragma unroll
-        for (int k = 0; k < BK / 16; ++k) {
-          const uint64_t da = make_desc_k_sw128(a_addr + k * 32);
-          umma_bf16_pair(tmem_base, da, make_desc_k_sw128(b_addr + k * 32), idesc1, (kb | k) != 0);
-          if (n2 > 0)
-            umma_bf16_pair(tmem_base + 256u, da, make_desc_k_sw128(b_addr + h1 * (BK * 2) + k * 32), idesc2, (kb | k) != 0);
-        }
-        umma_commit_pair(&empty[s], 3);
-      }
-      if (ok) umma_commit_pair(acc_full, 3);
-    }
-  } else {
-    lstm_tile_epilogue(p, tmem_base, acc_full, M, m0, n0, nu, warp, lane);
-  }
-  tc_fence_before();
-  __syncthreads();
-  cluster_sync_all();                                    // the peer's MMAs read this CTA's shared memory until they are done
-  if (warp == 1) tmem_dealloc_pair(tmem_base, 512);
-}
-
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -602,8 +486,6 @@ int gemm_bf16_setup() {
   cudaError_t e4 = cudaFuncSetAttribute(gemm_bf16_kernel<128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<128>::kSmem);
   cudaError_t e6 = cudaFuncSetAttribute(gemm_bf16_kernel<64, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<64>::kSmem);
   if (e6 != cudaSuccess) return TW_ERR_CUDA;
-  cudaError_t e7 = cudaFuncSetAttribute(gemm_lstm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairSmem);
-  if (e7 != cudaSuccess) return TW_ERR_CUDA;
   cudaError_t e5 = cudaFuncSetAttribute(gemm_lstm_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kWideSmem);
   return (e1 == cudaSuccess && e2 == cudaSuccess && e3 == cudaSuccess && e4 == cudaSuccess && e5 == cudaSuccess) ? TW_OK : TW_ERR_CUDA;
 }
@@ -619,7 +501,7 @@ static int sm_count() {
 }
 
 bool launch_gemm_lstm_wide(const CUtensorMap& tmA, const CUtensorMap& tmB64, const CUtensorMap& tmB32,
-                           const GemmBf16Params& p, cudaStream_t st, const CUtensorMap* tmB16) {
+                           const GemmBf16Params& p, cudaStream_t st) {
   if (p.epi != 1 || p.M <= 0 || p.N <= 0 || (p.N & 31) != 0) return false;
   const int num_sms = sm_count();
   const int mt = (p.M + BM - 1) / BM, nt256 = (p.N + 255) / 256;
@@ -628,24 +510,6 @@ bool launch_gemm_lstm_wide(const CUtensorMap& tmA, const CUtensorMap& tmB64, con
   if (n_split < 1) return false;
   const int units = p.N >> 5;
   if (((units + n_split - 1) / n_split) * 32 > kWideMaxBN) return false;
-  static const bool use_pairs = [] { const char* e = getenv("TW_GEMM_PAIRS"); return e != nullptr && e[0] == '1'; }();
-  if (use_pairs && tmB16 != nullptr) {
-    // CTA pairs: row tiles in pairs, the pair's columns split over floor((grid / 2) / row pairs) pairs
-    const int mp = (p.M + 2 * BM - 1) / (2 * BM), pairs = num_sms / 2;
-    const int nsp = pairs / mp;
-    if (nsp >= 1 && ((units + nsp - 1) / nsp) * 32 <= kWideMaxBN) {
-      cudaLaunchConfig_t cfg = {};
-      cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(kThreadsWide); cfg.dynamicSmemBytes = kPairSmem; cfg.stream = st;
-      cudaLaunchAttribute attr[2];
-      attr[0].id = cudaLaunchAttributeClusterDimension;
-      attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-      attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-      attr[1].val.programmaticStreamSerializationAllowed = 1;
-      cfg.attrs = attr; cfg.numAttrs = g_pdl_on ? 2 : 1;
-      if (cudaLaunchKernelEx(&cfg, gemm_lstm_pair_kernel, tmA, tmB64, tmB32, *tmB16, p) == cudaSuccess) return true;
-      cudaGetLastError();
-    }
-  }
   // one CTA per SM: the kernel splits the columns of each row tile over floor(grid / row tiles of this launch) CTAs
   launch_pdl(gemm_lstm_wide_kernel, dim3(num_sms), dim3(kThreadsWide), kWideSmem, st, tmA, tmB64, tmB32, p);
   return true;

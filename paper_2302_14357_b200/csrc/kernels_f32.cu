@@ -203,7 +203,7 @@ __global__ void __launch_bounds__(256) expand_f32_kernel(const float* __restrict
   const int R = R_dev ? *R_dev : R_max;
   const int r = blockIdx.x;
   if (r >= R) return;
-  const int sl = row_slen ? row_slen[r] : S;
+  const int sl = row_slen ? min(max(row_slen[r], 0), S) : S;   // a caller's value outside [0, S] must not index past the row
   const float* lp = logp + (long long)r * S * V;
   if (threadIdx.x == 0) {
     // the recursion is S steps long and its values grow to hundreds of nats: carry it in float64
@@ -276,11 +276,12 @@ __global__ void __launch_bounds__(256) expand_f32_kernel(const float* __restrict
   }
 }
 
-__global__ void rows_from_groups_kernel(const int* row_group, const int* seg_len, int R, int S,
+__global__ void rows_from_groups_kernel(const int* row_group, const int* seg_len, int R, int G, int S,
                                         int* row_e0, int* row_slen) {
   int r = blockIdx.x * blockDim.x + threadIdx.x;
   if (r >= R) return;
   int g = row_group[r];
+  if (g < 0 || g >= G) { row_e0[r] = 0; row_slen[r] = 0; return; }   // no such segment: an empty row, nothing is read for it
   row_e0[r] = g * S;
   int sl = seg_len ? seg_len[g] : S;
   row_slen[r] = sl < 0 ? 0 : (sl > S ? S : sl);
@@ -320,10 +321,10 @@ void launch_expand_f32(const float* logp, const float* ld_old, const int* row_sl
                                            ldnb, la, ldphi_d, la_d, cand);
 }
 
-void launch_rows_from_groups(const int* row_group, const int* seg_len, int R, int S, int* row_e0,
+void launch_rows_from_groups(const int* row_group, const int* seg_len, int R, int G, int S, int* row_e0,
                              int* row_slen, cudaStream_t st) {
   if (R <= 0) return;
-  rows_from_groups_kernel<<<(R + 255) / 256, 256, 0, st>>>(row_group, seg_len, R, S, row_e0, row_slen);
+  rows_from_groups_kernel<<<(R + 255) / 256, 256, 0, st>>>(row_group, seg_len, R, G, S, row_e0, row_slen);
 }
 
 }  // namespace tw

@@ -35,7 +35,7 @@ int scratch_for_current_device(float** out) {
 }  // namespace
 
 extern "C" int tw_joiner_expand_noalloc(const float* W_out, const float* b_out, int32_t J, int32_t V,
-                                        int32_t S, int32_t blank, const float* E_seg, const float* Pp,
+                                        int32_t S, int32_t blank, int32_t joiner_act, const float* E_seg, const float* Pp,
                                         const int32_t* row_group, const int32_t* seg_len,
                                         const float* ld_old, int32_t G, int32_t R, float* out_ldphi,
                                         float* out_ldnb, float* out_la, void* stream) {
@@ -44,6 +44,7 @@ extern "C" int tw_joiner_expand_noalloc(const float* W_out, const float* b_out, 
     return TW_ERR_ARG;
   if (J < 1 || V < 2 || S < 1 || S > TW_MAX_SEGMENT || blank < 0 || blank >= V || G < 0 || R < 0)
     return TW_ERR_ARG;
+  if (joiner_act != TW_ACT_TANH && joiner_act != TW_ACT_RELU) return TW_ERR_ARG;
   if (R > kMaxRows || (long long)R * S * V > kScratchFloats) return TW_ERR_LIMIT;
   if (R == 0) return TW_OK;
   float* scratch = nullptr;
@@ -55,10 +56,10 @@ extern "C" int tw_joiner_expand_noalloc(const float* W_out, const float* b_out, 
   cudaStream_t st = (cudaStream_t)stream;
   // every element of the scratch that is read below is written first by this call, so nothing left by
   // an earlier call can leak in and nothing needs clearing
-  launch_rows_from_groups(row_group, seg_len, R, S, row_e0, row_slen, st);
+  launch_rows_from_groups(row_group, seg_len, R, G, S, row_e0, row_slen, st);
   JoinerRows jr{};
   jr.E = E_seg; jr.row_e0 = row_e0; jr.Pp = Pp; jr.row_p = nullptr; jr.row_slen = row_slen;
-  jr.R_dev = nullptr; jr.R_max = R; jr.S = S; jr.J = J; jr.V = V;
+  jr.R_dev = nullptr; jr.R_max = R; jr.S = S; jr.J = J; jr.V = V; jr.act = joiner_act;
   launch_joiner_f32(jr, W_out, b_out, logp, st);
   launch_log_softmax(jr, blank, logp, st);
   launch_expand_f32(logp, ld_old, row_slen, nullptr, R, S, V, blank, out_ldphi, out_ldnb, out_la, nullptr,

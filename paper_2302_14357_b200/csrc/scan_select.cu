@@ -53,7 +53,7 @@ __global__ void __launch_bounds__(kMaxT) scan_select_kernel(ScanSelectArgs a) {
   const int r = blockIdx.x;
   if (r >= R) return;
   const int S = a.S, V = a.V, blank = a.blank;
-  const int sl = a.dnb_in ? 1 : (a.row_slen ? a.row_slen[r] : S);
+  const int sl = a.dnb_in ? 1 : (a.row_slen ? min(max(a.row_slen[r], 0), S) : S);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int kT = blockDim.x, nwarps = kT >> 5;
   const int gshift = kT >= 256 ? 4 : 3, ngroups = kT >> gshift;   // groups of 16 threads (8 in a 128-thread CTA): at least 16 groups

@@ -1,5 +1,4 @@
 // C ABI of libtw: handle life-cycle, the decode driver and the separately callable stages.
-#include <stdlib.h>
 #include <new>
 #include <vector>
 #include <stdio.h>
@@ -51,7 +50,6 @@ int make_bf16_mat(tw_handle* h, Bf16Mat* m, const float* src, long long rows, lo
     TW_TRY(make_tmap_bf16(&m->as_B256, m->ptr, rows, K, 256));
     TW_TRY(make_tmap_bf16(&m->as_B64, m->ptr, rows, K, 64));
     TW_TRY(make_tmap_bf16(&m->as_B32, m->ptr, rows, K, 32));
-    TW_TRY(make_tmap_bf16(&m->as_B16, m->ptr, rows, K, 16));
   }
   return TW_OK;
 }
@@ -95,7 +93,7 @@ void enqueue_predictor(tw_handle* h, const int* tok, const float* hc_in, const i
       p.epi = 1;
       p.lstm = LstmEpi{hc_in, idx_in, hc_out, idx_out, L, l, Hd,
                        (l + 1 < L) ? h->bf.X[l + 1].ptr : h->bf.Htop.ptr, (l + 1 < L) ? 2LL * Hd : (long long)Hd};
-      if (!launch_gemm_lstm_wide(h->bf.X[l].as_A, h->bf.W_cat[l].as_B64, h->bf.W_cat[l].as_B32, p, st, &h->bf.W_cat[l].as_B16))
+      if (!launch_gemm_lstm_wide(h->bf.X[l].as_A, h->bf.W_cat[l].as_B64, h->bf.W_cat[l].as_B32, p, st))
         launch_gemm_bf16(h->bf.X[l].as_A, h->bf.W_cat[l].as_B128, h->bf.W_cat[l].as_B256, p, st);
     }
     gemm_bf16(h, h->bf.Htop, h->bf.W_p, n_dev, n_max, Pp_out, idx_out, h->J, nullptr, st);
@@ -253,8 +251,7 @@ int build_bf16(tw_handle* h) {
     h->hs_fused.dnb_sel = h->bf.ldnb_pad;        // the step's hyp_step_kernel picks the rows' best tokens itself
     h->hs_fused.V = h->bf.Vp;                    // row pitch of delta_nb there (padding columns hold 0)
     // hyp_step_kernel builds the predictor's work list and operand rows itself (HypState::inline_gather)
-    const char* ig = getenv("TW_INLINE_GATHER");
-    if (h->hs_fused.defer_rows && h->pred_kind != TW_PRED_STATELESS && !(ig && ig[0] == '0')) {
+    if (h->hs_fused.defer_rows && h->pred_kind != TW_PRED_STATELESS) {
       h->hs_fused.inline_gather = 1;
       for (int l = 0; l < h->L; ++l) {
         h->hs_fused.xg_dst[l] = h->bf.X[l].ptr; h->hs_fused.xg_ld[l] = (int)h->bf.X[l].K; h->hs_fused.xg_off[l] = (l == 0) ? 0 : h->Hd;
@@ -544,6 +541,21 @@ int tw_set_monotonic(tw_handle* h, int on) {
   return TW_OK;
 }
 
+int tw_set_inline_gather(tw_handle* h, int on) {
+  if (!h) return TW_ERR_ARG;
+  if (h->stream_B > 0) return TW_ERR_STATE;
+  tw_handle* all[3] = {h, h->lane[0], h->lane[1]};
+  for (tw_handle* x : all) {
+    if (!x) continue;
+    // the operand rows' addresses were filled in by tw_init whenever the fused decode path with an LSTM predictor exists
+    const bool can = x->mode == TW_MODE_BF16 && x->bf.fused_ok && x->hs_fused.defer_rows && x->pred_kind != TW_PRED_STATELESS;
+    if (on && !can) return TW_ERR_STATE;
+    if (can) x->hs_fused.inline_gather = on ? 1 : 0;
+    if (x->graph_exec) { cudaGraphExecDestroy(x->graph_exec); x->graph_exec = nullptr; }   // captured arguments are by value
+  }
+  return TW_OK;
+}
+
 int tw_set_lanes(tw_handle* h, int on) {
   if (!h) return TW_ERR_ARG;
   h->lanes_on = on != 0;
@@ -559,6 +571,7 @@ int tw_set_graph(tw_handle* h, int on) {
 int tw_set_profiling(tw_handle* h, int on) {
   if (!h) return TW_ERR_ARG;
   h->profiling = on != 0;
+  h->stats.ns_joiner = h->stats.ns_scan = h->stats.joiner_launches = 0;   // the stage calls add to these while it is on
   return TW_OK;
 }
 
@@ -584,6 +597,24 @@ const char* tw_strerror(int s) {
 }
 
 }  // extern "C"
+
+namespace {
+enum Stage { kStStart = -1, kStPrologue = 0, kStPredictor, kStJoiner, kStScan, kStHyp, kStCount };
+
+// Profiling: records an event that closes stage `stage` (the time since the previous mark is its).
+void mark(tw_handle* h, int stage, cudaStream_t st) {
+  if (!h->profiling) return;
+  const size_t i = h->marks.size();
+  if (i >= h->events.size()) {
+    cudaEvent_t e;
+    if (cudaEventCreate(&e) != cudaSuccess) { h->profiling = false; return; }
+    h->events.push_back(e);
+  }
+  cudaEventRecord(h->events[i], st);
+  h->marks.push_back(stage);
+}
+
+}  // namespace
 
 #include "tw_api_stages.inc"
 #include "tw_api_decode.inc"

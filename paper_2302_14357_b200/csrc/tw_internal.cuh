@@ -125,8 +125,9 @@ struct ScanSelectArgs {
 bool scan_select_fits(int S, int V);   // the row's S x V logits fit in shared memory
 int scan_select_setup();
 void launch_scan_select(const ScanSelectArgs& a, bool fast_math, cudaStream_t st);
-// helper for the stage entry points: row_e0[r] = row_group[r] * S, row_slen[r] = seg_len[row_group[r]]
-void launch_rows_from_groups(const int* row_group, const int* seg_len, int R, int S, int* row_e0,
+// helper for the stage entry points: row_e0[r] = row_group[r] * S, row_slen[r] = seg_len[row_group[r]] clamped to
+// [0, S]; a row whose group is outside [0, G) becomes an empty row (length 0)
+void launch_rows_from_groups(const int* row_group, const int* seg_len, int R, int G, int S, int* row_e0,
                              int* row_slen, cudaStream_t st);
 
 // ---------------------------------------------------------------------------------------------

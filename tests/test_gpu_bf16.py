@@ -58,11 +58,11 @@ def test_joiner_segment_bf16(V, J, S, R):
     assert worst < BF16_STAGE_TOL, worst
 
 
-@pytest.mark.parametrize("layers,hidden,R", [(1, 64, 9), (2, 128, 9), (2, 1024, 1200), (1, 640, 1800)])
+@pytest.mark.parametrize("layers,hidden,R", [(1, 64, 9), (2, 128, 9), (2, 1024, 1200), (2, 1024, 1280), (1, 640, 1800), (3, 512, 700)])
 def test_predictor_step_bf16(layers, hidden, R):
-    """One predictor step per row against the oracle's LSTM.  The two large cases have more 128 x 256 gate
-    tiles than the device has SMs, which selects the single-wave gate GEMM (tiles of 256, 288 and 320
-    columns, a ragged last row tile); a sample of their rows is checked."""
+    """One predictor step per row against the oracle's LSTM, every row and every element.  The large cases
+    have more 128 x 256 gate tiles than the device has SMs, which selects the single-wave gate GEMM (tiles of
+    256, 288 and 320 columns, ragged and full last row tiles)."""
     cfg = _cfg(layers=layers, hidden=hidden)
     m, dec = _decoder(cfg, 2, max_batch=(R + 3) // 4)
     om = oracle_model(m)
@@ -72,14 +72,10 @@ def test_predictor_step_bf16(layers, hidden, R):
     out, Pp = dec.predictor_step(tokens, state)
     out, Pp = out.cpu().numpy(), Pp.cpu().numpy()
     assert np.all(np.isfinite(out)) and np.all(np.isfinite(Pp))
-    rows = range(R) if R <= 64 else sorted(set([0, 1, 127, 128, R - 2, R - 1]) | set(rng.integers(0, R, size=18).tolist()))
-    for r in rows:
-        st = ([state[r, l, 0].astype(np.float64) for l in range(layers)], [state[r, l, 1].astype(np.float64) for l in range(layers)])
-        (h, c), o = rm.lstm_step(om, st, int(tokens[r]))
-        for l in range(layers):
-            np.testing.assert_allclose(out[r, l, 0], h[l], atol=BF16_STAGE_TOL)
-            np.testing.assert_allclose(out[r, l, 1], c[l], atol=BF16_STAGE_TOL)
-        np.testing.assert_allclose(Pp[r], om.W_p @ o, atol=BF16_STAGE_TOL)
+    h, c, o = rm.lstm_step_rows(om, state[:, :, 0], state[:, :, 1], tokens)
+    np.testing.assert_allclose(out[:, :, 0], h, rtol=0, atol=BF16_STAGE_TOL)
+    np.testing.assert_allclose(out[:, :, 1], c, rtol=0, atol=BF16_STAGE_TOL)
+    np.testing.assert_allclose(Pp, o @ om.W_p.T, rtol=0, atol=BF16_STAGE_TOL)
 
 
 @pytest.mark.parametrize("V,J,S,R", [(256, 64, 3, 5), (256, 128, 1, 40), (1024, 640, 3, 45), (4096, 1024, 2, 70),
@@ -243,22 +239,29 @@ def _top1_agreement(cfg, S, batch, T):
         got = nbest_from_arrays(tokens, olens, scores, b)
         ref, _ = tws.token_wise_beam_search(om, enc[b, :lens[b]], cfg.N, S, max_iters=4 * S + 16)
         agree += got[0][0] == ref[0][0]
-        gaps.append(abs(got[0][1] - ref[0][1]))
+        if got[0][0] == ref[0][0]:
+            gaps.append(abs(got[0][1] - ref[0][1]))
         assert len(got) == len(ref) and status[b] == 0
-    return agree / batch, max(gaps), dec.stats()
+    return agree, max(gaps, default=0.0), dec.stats()
+
+
+# The bar of the bf16 end-to-end tests: the best hypothesis is the oracle's for all sampled utterances but at most
+# one (a near-tie between the two best sequences may legitimately fall the other way at bf16 precision), and where
+# the sequences agree the scores are within TOP1_GAP nats (stage tolerance 2e-2 per pass, errors of random sign)
+TOP1_GAP = 0.05
 
 
 def test_decode_bf16_small_model_top1():
-    rate, gap, st = _top1_agreement(_cfg(batch=6, T=40), 3, 6, 40)
-    print("bf16 top-1 agreement %.2f, max top-1 score gap %.3g" % (rate, gap))
-    assert rate >= 0.5 and gap < 0.5
+    agree, gap, st = _top1_agreement(_cfg(batch=6, T=40), 3, 6, 40)
+    print("bf16 top-1 agreement %d/6, max top-1 score gap %.3g" % (agree, gap))
+    assert agree >= 5 and gap < TOP1_GAP
 
 
-@pytest.mark.parametrize("name,S,batch,T", [("c1", 3, 4, 80), ("c3", 3, 2, 45), ("p1", 3, 4, 60), ("p1", 5, 2, 50)])
+@pytest.mark.parametrize("name,S,batch,T", [("c1", 3, 6, 80), ("c3", 3, 4, 45), ("p1", 3, 6, 60), ("p1", 5, 4, 50)])
 def test_decode_bf16_config_shapes_top1(name, S, batch, T):
-    rate, gap, st = _top1_agreement(tw_synth.get_config(name), S, batch, T)
-    print("%s bf16 top-1 agreement %.2f, max top-1 score gap %.3g" % (name, rate, gap))
-    assert rate >= 0.5 and gap < 1.0
+    agree, gap, st = _top1_agreement(tw_synth.get_config(name), S, batch, T)
+    print("%s bf16 top-1 agreement %d/%d, max top-1 score gap %.3g" % (name, agree, batch, gap))
+    assert agree >= batch - 1 and gap < TOP1_GAP
     assert st["calls"] > 0
 
 
@@ -266,8 +269,8 @@ def test_decode_bf16_config_shapes_top1(name, S, batch, T):
 def test_decode_bf16_paper_shape_small_beams(N):
     """The paper's tables also use beams of 1 and 2: greedy-sized lists on the paper-shaped workload."""
     cfg = tw_synth.get_config("p1").with_(N=N)
-    rate, gap, st = _top1_agreement(cfg, 3, 4, 60)
-    assert rate >= 0.5 and gap < 1.0
+    agree, gap, st = _top1_agreement(cfg, 3, 4, 60)
+    assert agree >= 3 and gap < TOP1_GAP
     assert st["calls"] > 0 and st["fused_on"] == 1
 
 
@@ -295,49 +298,18 @@ def test_repeated_decodes_are_bit_identical():
     dec.close()
 
 
-def test_cta_pair_gate_gemm_matches_single_cta_kernel(tmp_path):
-    """TW_GEMM_PAIRS=1 runs the LSTM gate GEMMs on CTA pairs (tcgen05 cta_group::2).  The switch is read once per
-    process, so the pair run is a child process; both runs accumulate K in the same order."""
-    import os, subprocess, sys
-    code = """
-import sys, numpy as np, tw_synth
-sys.path.insert(0, 'tests')
-from paper_2302_14357_b200.binding import MODE_BF16, TwDecoder, weights_from_synth
-cfg = tw_synth.WorkloadConfig('b', 4, 30, (15, 30), 64, 'lstm', 64, 2, 1024, 128, 256, 3.0, 4, (3,), 'bf16', 3)
-m = tw_synth.make_model(cfg)
-R = 1200
-dec = TwDecoder(weights_from_synth(m), N=4, S=2, mode=MODE_BF16, max_batch=R // 4, max_T=30)
-rng = np.random.default_rng(4)
-tokens = rng.integers(0, cfg.V, size=R).astype(np.int32)
-state = (rng.standard_normal((R, 2, 2, 1024)) * 0.5).astype(np.float32)
-out, Pp = dec.predictor_step(tokens, state)
-np.savez(sys.argv[1], out=out.cpu().numpy(), Pp=Pp.cpu().numpy())
-"""
-    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-    res = {}
-    for name, flag in (("single", "0"), ("pair", "1")):
-        path = str(tmp_path / (name + ".npz"))
-        env = dict(os.environ, TW_GEMM_PAIRS=flag, PYTHONPATH=root)
-        r = subprocess.run([sys.executable, "-c", code, path], env=env, cwd=root, capture_output=True, text=True, timeout=300)
-        assert r.returncode == 0, r.stderr[-2000:]
-        res[name] = np.load(path)
-    assert np.all(np.isfinite(res["pair"]["out"]))
-    np.testing.assert_allclose(res["pair"]["out"], res["single"]["out"], rtol=0, atol=1e-5)
-    np.testing.assert_allclose(res["pair"]["Pp"], res["single"]["Pp"], rtol=0, atol=1e-4)
-
-
-def test_work_list_built_by_hyp_step_equals_gather_kernel(monkeypatch):
+def test_work_list_built_by_hyp_step_equals_gather_kernel():
     """Fused bf16 decode: the predictor's work list and operand rows written by hyp_step_kernel (entries in an
     order that varies between runs) give the same decode, bit for bit, as the gather kernel's deterministic
-    list (TW_INLINE_GATHER=0, read by tw_init).  A ragged batch with a 2-layer LSTM, in both search variants."""
+    list (tw_set_inline_gather(h, 0)).  A ragged batch with a 2-layer LSTM, in both search variants."""
     from paper_2302_14357_b200.binding import MODE_BF16, TwDecoder, weights_from_synth
     cfg = tw_synth.WorkloadConfig("ig", 24, 60, (20, 60), 64, "lstm", 64, 2, 128, 128, 512, 3.0, 5, (3,), "bf16", 17)
     m = tw_synth.make_model(cfg)
     enc, lens = tw_synth.make_encoder_batch(cfg)
     runs = {}
     for flag in ("1", "0"):
-        monkeypatch.setenv("TW_INLINE_GATHER", flag)
         dec = TwDecoder(weights_from_synth(m), N=cfg.N, S=3, mode=MODE_BF16, max_batch=cfg.batch, max_T=cfg.T)
+        dec.set_inline_gather(flag == "1")
         out = []
         for mono in (False, True):
             dec.set_monotonic(mono)

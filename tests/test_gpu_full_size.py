@@ -8,6 +8,9 @@ from helpers import check_against_oracle, nbest_from_arrays, oracle_model
 from oracle import token_wise_search as tws
 
 pytestmark = pytest.mark.gpu
+# bf16 end to end: the oracle's best sequence for all sampled utterances but at most one (a near-tie may fall the
+# other way at bf16 precision); where the sequences agree, scores within TOP1_GAP nats
+TOP1_GAP = 0.05
 
 
 def _decode(cfg, S, mode, T=None):
@@ -46,19 +49,20 @@ def test_full_batch_fp32_sampled_utterances(name, S, sample, T):
 
 def test_full_batch_bf16_c3_top1_sampled():
     cfg = tw_synth.get_config("c3")
-    S, T = 3, 240
+    S, T = 3, 150
     m, enc, lens, (tokens, olens, scores, status), st = _decode(cfg, S, 1, T)
     assert st["limit_hits"] == 0
     om = oracle_model(m)
     agree = 0
-    sample = (1, 64, 127)
+    sample = (0, 1, 17, 40, 64, 65, 99, 127)
     for b in sample:
         got = nbest_from_arrays(tokens, olens, scores, b)
         ref, _ = tws.token_wise_beam_search(om, enc[b, :lens[b]], cfg.N, S, max_iters=4 * S + 16)
         agree += got[0][0] == ref[0][0]
-        assert abs(got[0][1] - ref[0][1]) < 1.0
+        if got[0][0] == ref[0][0]:
+            assert abs(got[0][1] - ref[0][1]) < TOP1_GAP
     print("c3 bf16 top-1 agreement on sampled utterances: %d/%d" % (agree, len(sample)))
-    assert agree >= 2
+    assert agree >= len(sample) - 1
 
 
 def test_full_batch_bf16_c4_two_lanes_ragged_sampled():
@@ -81,11 +85,12 @@ def test_full_batch_bf16_c4_two_lanes_ragged_sampled():
     assert st["limit_hits"] == 0 and np.all(status == 0)
     assert st["frames"] == int(lens.sum()) and np.all(np.diff(scores, axis=1) <= 0)
     om = oracle_model(m)
-    agree, sample = 0, (7, 255, 300)
+    agree, sample = 0, (7, 255, 256, 300, 511)
     for b in sample:
         got = nbest_from_arrays(tokens, olens, scores, b)
         ref, _ = tws.token_wise_beam_search(om, enc[b, :lens[b]], cfg.N, S, max_iters=4 * S + 16)
         agree += got[0][0] == ref[0][0]
-        assert abs(got[0][1] - ref[0][1]) < 1.0
+        if got[0][0] == ref[0][0]:
+            assert abs(got[0][1] - ref[0][1]) < TOP1_GAP
     print("c4 bf16 top-1 agreement on sampled utterances: %d/%d" % (agree, len(sample)))
-    assert agree >= 2
+    assert agree >= len(sample) - 1

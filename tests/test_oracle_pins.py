@@ -118,6 +118,43 @@ def test_lstm_predictor_matches_library_lstm(layers):
     np.testing.assert_allclose(o2, o, atol=0)
 
 
+@pytest.mark.parametrize("layers", [1, 3])
+def test_lstm_step_rows_matches_library_lstm_cell_batch(layers):
+    """The batched predictor step against torch.nn.LSTM run on a batch with given (h0, c0) (fp64, CPU), and
+    against the one-row step: a transposed weight, a swapped gate or a mixed-up row would fail."""
+    torch = pytest.importorskip("torch")
+    rng = np.random.default_rng(11)
+    V, E, Hd, R = 7, 5, 6, 9
+    W_ih = [rng.standard_normal((4 * Hd, E if l == 0 else Hd)) for l in range(layers)]
+    W_hh = [rng.standard_normal((4 * Hd, Hd)) for l in range(layers)]
+    b = [rng.standard_normal(4 * Hd) for l in range(layers)]
+    emb = rng.standard_normal((V, E))
+    model = rm.RnntModel(W_e=np.zeros((2, 3)), W_p=np.zeros((2, Hd)), W_out=np.zeros((V, 2)),
+                         b_out=np.zeros(V), emb=emb, lstm_W_ih=W_ih, lstm_W_hh=W_hh, lstm_b=b)
+    h0, c0 = rng.standard_normal((R, layers, Hd)), rng.standard_normal((R, layers, Hd))
+    tokens = rng.integers(0, V, size=R)
+    h1, c1, out = rm.lstm_step_rows(model, h0, c0, tokens)
+    lib = torch.nn.LSTM(E, Hd, num_layers=layers).double()
+    with torch.no_grad():
+        for l in range(layers):
+            getattr(lib, f"weight_ih_l{l}").copy_(torch.from_numpy(W_ih[l]))
+            getattr(lib, f"weight_hh_l{l}").copy_(torch.from_numpy(W_hh[l]))
+            getattr(lib, f"bias_ih_l{l}").copy_(torch.from_numpy(b[l]))
+            getattr(lib, f"bias_hh_l{l}").zero_()
+        o_lib, (h_lib, c_lib) = lib(torch.from_numpy(emb[tokens]).unsqueeze(0),
+                                    (torch.from_numpy(h0.transpose(1, 0, 2).copy()), torch.from_numpy(c0.transpose(1, 0, 2).copy())))
+    np.testing.assert_allclose(out, o_lib[0].numpy(), atol=1e-12)
+    np.testing.assert_allclose(h1, h_lib.numpy().transpose(1, 0, 2), atol=1e-12)
+    np.testing.assert_allclose(c1, c_lib.numpy().transpose(1, 0, 2), atol=1e-12)
+    for r in range(R):
+        st = ([h0[r, l] for l in range(layers)], [c0[r, l] for l in range(layers)])
+        (h, c), o = rm.lstm_step(model, st, int(tokens[r]))
+        np.testing.assert_allclose(out[r], o, atol=1e-12)
+        for l in range(layers):
+            np.testing.assert_allclose(h1[r, l], h[l], atol=1e-12)
+            np.testing.assert_allclose(c1[r, l], c[l], atol=1e-12)
+
+
 def test_stateless_predictor_is_embedding_of_last_token():
     emb = np.arange(12.0).reshape(4, 3)
     model = rm.RnntModel(np.zeros((2, 2)), np.zeros((2, 3)), np.zeros((4, 2)), np.zeros(4), emb)
