@@ -4,7 +4,8 @@
  *
  * C ABI.  Conventions that hold for every call unless a comment says otherwise:
  *   - pointers are DEVICE pointers; a name starting with host_ is a HOST pointer;
- *   - matrices are dense, row-major, float32; int arrays are int32;
+ *   - matrices are dense, row-major, float32; int arrays are int32; the model's weights and the encoder frames
+ *     are float32 or bfloat16 as tw_model::dtype says (those parameters are `const void*`);
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream);
  *     work is enqueued on it and the call returns without synchronising, except
  *     where stated;
@@ -42,7 +43,8 @@ typedef enum {
   TW_ERR_TIMEOUT = 6 /* a bounded device-side wait gave up; results are not valid       */
 } tw_status;
 
-enum { TW_MODE_F32 = 0, TW_MODE_BF16 = 1 };
+enum { TW_MODE_F32 = 0, TW_MODE_BF16 = 1 };   /* arithmetic of the decoder (tw_config::mode)                   */
+enum { TW_F32 = 0, TW_BF16 = 1 };             /* element type of the caller's weights and frames (tw_model::dtype) */
 enum { TW_PRED_STATELESS = 0, TW_PRED_LSTM = 1 };
 enum { TW_ACT_TANH = 0, TW_ACT_RELU = 1 };   /* joiner hidden nonlinearity */
 
@@ -56,23 +58,36 @@ enum { TW_ACT_TANH = 0, TW_ACT_RELU = 1 };   /* joiner hidden nonlinearity */
  *   predictor: stateless  g = emb[last token]         (P == emb_dim; empty prefix -> emb[blank])
  *              LSTM       lstm_layers stacked cells, gate order (input, forget, cell, output),
  *                         one bias per layer, g = top layer's h   (P == lstm_hidden);
- *                         InitPredictor() = one step on the blank token from an all-zero state.
- * Weight pointers are device float32; in TW_MODE_BF16 the library keeps bf16 copies (exact if the
- * values are already bf16-representable).  The per-layer pointer tables are HOST arrays of device
- * pointers.  Nothing passed here is referenced after tw_init returns.
+ *                         InitPredictor(): see pred_init_* below.
+ * dtype says what the weight pointers, pred_init_* and every encoder-frame argument of this handle point to:
+ * TW_F32 (float32) or TW_BF16 (bfloat16, 2 bytes per element).  It is independent of tw_config::mode: the
+ * library keeps float32 copies for its float32 kernels and, in TW_MODE_BF16, bfloat16 copies for the tensor
+ * cores (exact if the values are bfloat16-representable, as they are when dtype is TW_BF16).  The per-layer
+ * pointer tables are HOST arrays of device pointers.  Nothing passed here is referenced after tw_init returns.
+ *
+ * InitPredictor() (Sec. 3.2: the predictor's initial state is a learned quantity, initialised like a weight).
+ * Both fields are optional; with both NULL the initial state is one predictor step on the blank token from an
+ * all-zero state (LSTM) or the blank token's embedding (stateless).
+ *   pred_init_state  [lstm_layers, 2, lstm_hidden]  per layer h then c (LSTM only; NULL: zeros when
+ *                    pred_init_out is given)
+ *   pred_init_out    [P]  the predictor output of the empty token prefix (NULL with a state given: the top
+ *                    layer's h)
  */
 typedef struct {
   int32_t D_enc, P, J, V, blank;
   int32_t pred_kind, emb_dim, lstm_layers, lstm_hidden;
   int32_t joiner_act; /* TW_ACT_TANH or TW_ACT_RELU */
-  const float* W_e;   /* [J, D_enc] */
-  const float* W_p;   /* [J, P]     */
-  const float* W_out; /* [V, J]     */
-  const float* b_out; /* [V]        */
-  const float* emb;   /* [V, emb_dim] */
-  const float* const* host_lstm_W_ih; /* [lstm_layers] -> [4*Hd, in]  (in = emb_dim, then Hd) */
-  const float* const* host_lstm_W_hh; /* [lstm_layers] -> [4*Hd, Hd] */
-  const float* const* host_lstm_b;    /* [lstm_layers] -> [4*Hd]     */
+  int32_t dtype;      /* TW_F32 or TW_BF16 */
+  const void* W_e;   /* [J, D_enc] */
+  const void* W_p;   /* [J, P]     */
+  const void* W_out; /* [V, J]     */
+  const void* b_out; /* [V]        */
+  const void* emb;   /* [V, emb_dim] */
+  const void* const* host_lstm_W_ih; /* [lstm_layers] -> [4*Hd, in]  (in = emb_dim, then Hd) */
+  const void* const* host_lstm_W_hh; /* [lstm_layers] -> [4*Hd, Hd] */
+  const void* const* host_lstm_b;    /* [lstm_layers] -> [4*Hd]     */
+  const void* pred_init_state;       /* optional, see above */
+  const void* pred_init_out;         /* optional, see above */
 } tw_model;
 
 /*
@@ -122,8 +137,8 @@ int tw_destroy(tw_handle* h);
 
 /*
  * Algorithm 1 for a batch of B utterances, each decoded independently.
- *   enc      [B, T, D_enc]  encoder output (computed beforehand, Sec. 3.2); frames at or past
- *                           lengths[b] are ignored
+ *   enc      [B, T, D_enc]  encoder output (computed beforehand, Sec. 3.2), elements of the model's dtype;
+ *                           frames at or past lengths[b] are ignored
  *   lengths  [B]            0 <= lengths[b] <= T (values outside are clamped and flagged TW_ERR_ARG
  *                           in out_status[b])
  *   out_tokens [B, N, U_cap] N best token sequences, best first, padded with -1
@@ -136,7 +151,7 @@ int tw_destroy(tw_handle* h);
  * Returns TW_ERR_LIMIT if any utterance hit a cap (outputs are still valid for the others),
  * TW_ERR_ARG if B > max_batch, T > max_T or a pointer is null.
  */
-int tw_decode(tw_handle* h, const float* enc, const int32_t* lengths, int32_t B, int32_t T,
+int tw_decode(tw_handle* h, const void* enc, const int32_t* lengths, int32_t B, int32_t T,
               int32_t* out_tokens, int32_t* out_lens, double* out_scores, int32_t* out_status,
               void* stream);
 
@@ -146,7 +161,7 @@ int tw_decode(tw_handle* h, const float* enc, const int32_t* lengths, int32_t B,
  * and each chunk is decoded, as a streaming push, while the next one is on its way; the result is
  * the same as tw_decode's.  Pinned host memory is what makes the upload asynchronous.  Must not be
  * called while a streaming session is open on the handle. */
-int tw_decode_host(tw_handle* h, const float* host_enc, const int32_t* host_lengths, int32_t B,
+int tw_decode_host(tw_handle* h, const void* host_enc, const int32_t* host_lengths, int32_t B,
                    int32_t T, int32_t* host_out_tokens, int32_t* host_out_lens,
                    double* host_out_scores, int32_t* host_out_status, void* stream);
 
@@ -166,7 +181,7 @@ int tw_decode_host(tw_handle* h, const float* host_enc, const int32_t* host_leng
  * All four synchronise before returning.  TW_ERR_STATE without an open session.
  */
 int tw_stream_open(tw_handle* h, int32_t B, void* stream);
-int tw_stream_push(tw_handle* h, const float* enc_chunk, const int32_t* chunk_lens, int32_t Tc, void* stream);
+int tw_stream_push(tw_handle* h, const void* enc_chunk, const int32_t* chunk_lens, int32_t Tc, void* stream);
 int tw_stream_nbest(tw_handle* h, int32_t* out_tokens, int32_t* out_lens, double* out_scores,
                     int32_t* out_status, void* stream);
 int tw_stream_close(tw_handle* h, int32_t* out_tokens, int32_t* out_lens, double* out_scores,
@@ -178,9 +193,9 @@ int tw_max_tokens(const tw_handle* h);
 /*
  * Encoder half of the joiner's first layer, E = enc . W_e^T, computed once per frame
  * (Sec. 3.1 joiner; the split of the first layer is exact algebra).
- *   enc [rows, D_enc] -> out_E [rows, J]
+ *   enc [rows, D_enc] (the model's dtype) -> out_E [rows, J] float32
  */
-int tw_project_encoder(tw_handle* h, const float* enc, int32_t rows, float* out_E, void* stream);
+int tw_project_encoder(tw_handle* h, const void* enc, int32_t rows, float* out_E, void* stream);
 
 /*
  * J = Softmax(Joiner(seg, pred)) of Algorithm 1 for R hypothesis rows, in log space.

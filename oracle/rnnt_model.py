@@ -21,7 +21,8 @@ def _f64(x):
 class RnntModel:
     def __init__(self, W_e, W_p, W_out, b_out, emb,
                  lstm_W_ih: Sequence = (), lstm_W_hh: Sequence = (), lstm_b: Sequence = (),
-                 blank: int = 0, activation: str = "tanh"):
+                 blank: int = 0, activation: str = "tanh",
+                 pred_init_state=None, pred_init_out=None):
         self.W_e = _f64(W_e)        # [J, D_enc]
         self.W_p = _f64(W_p)        # [J, P]
         self.W_out = _f64(W_out)    # [V, J]
@@ -33,6 +34,10 @@ class RnntModel:
         self.blank = int(blank)
         assert activation in ("tanh", "relu")
         self.activation = activation
+        # InitPredictor() of Sec. 3.2 returns a learned initial state: optional here, as
+        # pred_init_state [L, 2, Hd] (per layer h then c) and / or pred_init_out [P]
+        self.pred_init_state = None if pred_init_state is None else _f64(pred_init_state)
+        self.pred_init_out = None if pred_init_out is None else _f64(pred_init_out)
         self.V = self.W_out.shape[0]
         assert self.W_e.shape[0] == self.W_p.shape[0] == self.W_out.shape[1]
         assert len(self.lstm_W_ih) == len(self.lstm_W_hh) == len(self.lstm_b)
@@ -105,12 +110,23 @@ def lstm_step_rows(model: RnntModel, h_prev: np.ndarray, c_prev: np.ndarray, tok
 
 
 def predictor_init(model: RnntModel):
-    """InitPredictor(): (state, output) for the empty token prefix."""
+    """InitPredictor(): (state, output) for the empty token prefix.  A model that carries a learned initial
+    state (Sec. 3.2) returns it: the state as given (zeros without one), the output as given (the top layer's
+    h without one).  Otherwise the blank token's embedding (stateless) or one step on the blank token from an
+    all-zero state (LSTM)."""
     if not model.is_lstm:
+        if model.pred_init_out is not None:
+            return None, model.pred_init_out.copy()
         return None, model.emb[model.blank].copy()
     L = len(model.lstm_W_ih)
     Hd = model.lstm_W_hh[0].shape[1]
     zero = ([np.zeros(Hd) for _ in range(L)], [np.zeros(Hd) for _ in range(L)])
+    if model.pred_init_state is not None or model.pred_init_out is not None:
+        st = zero
+        if model.pred_init_state is not None:
+            st = ([model.pred_init_state[l, 0].copy() for l in range(L)], [model.pred_init_state[l, 1].copy() for l in range(L)])
+        out = model.pred_init_out.copy() if model.pred_init_out is not None else st[0][L - 1].copy()
+        return st, out
     return lstm_step(model, zero, model.blank)
 
 

@@ -8,6 +8,7 @@ import numpy as np
 MODE_F32, MODE_BF16 = 0, 1
 PRED_STATELESS, PRED_LSTM = 0, 1
 ACT_TANH, ACT_RELU = 0, 1
+DT_F32, DT_BF16 = 0, 1
 TW_OK, TW_ERR_ARG, TW_ERR_ALLOC, TW_ERR_CUDA, TW_ERR_LIMIT, TW_ERR_STATE, TW_ERR_TIMEOUT = range(7)
 
 EXPORTED_SYMBOLS = [
@@ -30,8 +31,9 @@ class TwError(RuntimeError):
 
 
 class _Model(C.Structure):
-    _fields_ = [(n, C.c_int32) for n in ("D_enc", "P", "J", "V", "blank", "pred_kind", "emb_dim", "lstm_layers", "lstm_hidden", "joiner_act")] + \
-               [(n, C.c_void_p) for n in ("W_e", "W_p", "W_out", "b_out", "emb", "host_lstm_W_ih", "host_lstm_W_hh", "host_lstm_b")]
+    _fields_ = [(n, C.c_int32) for n in ("D_enc", "P", "J", "V", "blank", "pred_kind", "emb_dim", "lstm_layers", "lstm_hidden", "joiner_act", "dtype")] + \
+               [(n, C.c_void_p) for n in ("W_e", "W_p", "W_out", "b_out", "emb", "host_lstm_W_ih", "host_lstm_W_hh", "host_lstm_b",
+                                          "pred_init_state", "pred_init_out")]
 
 
 class _Config(C.Structure):
@@ -102,11 +104,14 @@ def _ptr(t) -> Optional[int]:
 
 
 class TwDecoder:
-    """A decoder handle (tw_init .. tw_destroy).  `weights` maps the tw_model field names to CUDA
-    float32 tensors ("lstm_W_ih", "lstm_W_hh", "lstm_b" are lists, one tensor per layer)."""
+    """A decoder handle (tw_init .. tw_destroy).  `weights` maps the tw_model field names to arrays or
+    tensors ("lstm_W_ih", "lstm_W_hh", "lstm_b" are lists, one per layer; "pred_init_state" and "pred_init_out"
+    are optional).  dtype "f32" or "bf16" is the element type in which the weights and, later, the encoder
+    frames are handed to the library (tw_model::dtype); values are converted to it here."""
 
     def __init__(self, weights: Dict, N: int, S: int, mode: int = MODE_F32, max_batch: int = 1, max_T: int = 1,
-                 max_iters_per_segment: int = 0, max_tokens: int = 0, blank: int = 0, joiner_act: str = "tanh"):
+                 max_iters_per_segment: int = 0, max_tokens: int = 0, blank: int = 0, joiner_act: str = "tanh",
+                 dtype: str = "f32"):
         import torch
         self._torch = torch
         self.lib = load_library()
@@ -114,9 +119,12 @@ class TwDecoder:
             raise RuntimeError("TwDecoder needs a CUDA device; there is no CPU path")
         self.device = torch.device("cuda", torch.cuda.current_device())
 
+        self.dtype = dtype
+        self._tdtype = {"f32": torch.float32, "bf16": torch.bfloat16}[dtype]
+
         def dev(x):
-            t = torch.as_tensor(x, dtype=torch.float32)
-            return t.to(self.device).contiguous()
+            t = torch.as_tensor(x) if not isinstance(x, np.ndarray) else torch.from_numpy(np.ascontiguousarray(x))
+            return t.to(self.device).to(self._tdtype).contiguous()
         weights = dict(weights)
         joiner_act = weights.pop("joiner_act", None) or joiner_act
         w = {k: ([dev(a) for a in v] if isinstance(v, (list, tuple)) else dev(v)) for k, v in weights.items() if v is not None}
@@ -132,6 +140,9 @@ class TwDecoder:
         m.emb_dim, m.lstm_layers = emb_dim, layers
         m.lstm_hidden = w["lstm_W_hh"][0].shape[1] if layers else 0
         m.joiner_act = {"tanh": ACT_TANH, "relu": ACT_RELU}[joiner_act]
+        m.dtype = {"f32": DT_F32, "bf16": DT_BF16}[dtype]
+        for name in ("pred_init_state", "pred_init_out"):
+            setattr(m, name, w[name].data_ptr() if name in w else None)
         for name in ("W_e", "W_p", "W_out", "b_out", "emb"):
             setattr(m, name, w[name].data_ptr())
         self._tables = []
@@ -163,6 +174,11 @@ class TwDecoder:
     def _f32(self, x):
         return self._torch.as_tensor(x, dtype=self._torch.float32, device=self.device).contiguous()
 
+    def _frames(self, x):
+        """Encoder frames on the device in the handle's element type."""
+        t = self._torch.as_tensor(x) if not isinstance(x, np.ndarray) else self._torch.from_numpy(np.ascontiguousarray(x))
+        return t.to(self.device).to(self._tdtype).contiguous()
+
     def _i32(self, x):
         return None if x is None else self._torch.as_tensor(x, dtype=self._torch.int32, device=self.device).contiguous()
 
@@ -179,9 +195,9 @@ class TwDecoder:
 
     # -- the calls of include/tw.h ------------------------------------------------------------
     def decode(self, enc, lengths):
-        """tw_decode: enc [B, T, D_enc] (CUDA float32), lengths [B] -> (tokens, lens, scores, status, rc)."""
+        """tw_decode: enc [B, T, D_enc], lengths [B] -> (tokens, lens, scores, status, rc)."""
         torch = self._torch
-        enc, lengths = self._f32(enc), self._i32(lengths)
+        enc, lengths = self._frames(enc), self._i32(lengths)
         B, T = enc.shape[0], enc.shape[1]
         tokens = torch.empty((B, self.N, self.U_cap), dtype=torch.int32, device=self.device)
         lens = torch.empty((B, self.N), dtype=torch.int32, device=self.device)
@@ -192,16 +208,25 @@ class TwDecoder:
         self._check(rc, "tw_decode", allow_limit=True)
         return tokens, lens, scores, status, rc
 
-    def decode_host(self, enc: np.ndarray, lengths: np.ndarray, out=None):
-        """tw_decode_host: host buffers in, host buffers out (copies are part of the call)."""
-        enc = np.ascontiguousarray(enc, dtype=np.float32)
+    def decode_host(self, enc, lengths: np.ndarray, out=None):
+        """tw_decode_host: host buffers in, host buffers out (copies are part of the call).  enc: a float32 numpy
+        array, or a CPU torch tensor of the handle's element type (numpy has no bfloat16)."""
+        if isinstance(enc, np.ndarray):
+            if self.dtype != "f32":
+                raise TypeError("a bf16 handle takes its host frames as a torch.bfloat16 CPU tensor")
+            enc = np.ascontiguousarray(enc, dtype=np.float32)
+            enc_ptr = enc.ctypes.data
+        else:
+            if enc.dtype != self._tdtype or enc.device.type != "cpu" or not enc.is_contiguous():
+                raise TypeError("host frames must be a contiguous CPU tensor of the handle's element type")
+            enc_ptr = enc.data_ptr()
         lengths = np.ascontiguousarray(lengths, dtype=np.int32)
         B, T = enc.shape[0], enc.shape[1]
         if out is None:
             out = (np.empty((B, self.N, self.U_cap), np.int32), np.empty((B, self.N), np.int32),
                    np.empty((B, self.N), np.float64), np.empty((B,), np.int32))
         tokens, lens, scores, status = out
-        rc = self.lib.tw_decode_host(self.h, enc.ctypes.data, lengths.ctypes.data, B, T, tokens.ctypes.data,
+        rc = self.lib.tw_decode_host(self.h, enc_ptr, lengths.ctypes.data, B, T, tokens.ctypes.data,
                                      lens.ctypes.data, scores.ctypes.data, status.ctypes.data, self._stream())
         self._check(rc, "tw_decode_host", allow_limit=True)
         return tokens, lens, scores, status, rc
@@ -219,7 +244,7 @@ class TwDecoder:
 
     def stream_push(self, enc_chunk, chunk_lens):
         """tw_stream_push: enc_chunk [B, Tc, D_enc], chunk_lens [B] valid frames of the chunk per utterance."""
-        enc_chunk, chunk_lens = self._f32(enc_chunk), self._i32(chunk_lens)
+        enc_chunk, chunk_lens = self._frames(enc_chunk), self._i32(chunk_lens)
         self._check(self.lib.tw_stream_push(self.h, enc_chunk.data_ptr(), chunk_lens.data_ptr(), enc_chunk.shape[1],
                                             self._stream()), "tw_stream_push", allow_limit=True)
 
@@ -235,7 +260,7 @@ class TwDecoder:
         return out + (rc,)
 
     def project_encoder(self, enc):
-        enc = self._f32(enc).reshape(-1, self.D_enc)
+        enc = self._frames(enc).reshape(-1, self.D_enc)
         out = self._torch.empty((enc.shape[0], self.J), dtype=self._torch.float32, device=self.device)
         self._check(self.lib.tw_project_encoder(self.h, enc.data_ptr(), enc.shape[0], out.data_ptr(), self._stream()), "tw_project_encoder")
         return out
@@ -315,7 +340,8 @@ def weights_from_synth(m) -> Dict:
     """tw_model fields from a tw_synth.SyntheticModel (plain attribute access, no arithmetic)."""
     return dict(W_e=m.W_e, W_p=m.W_p, W_out=m.W_out, b_out=m.b_out, emb=m.emb,
                 lstm_W_ih=list(m.lstm_W_ih), lstm_W_hh=list(m.lstm_W_hh), lstm_b=list(m.lstm_b),
-                joiner_act=m.cfg.joiner_act)
+                joiner_act=m.cfg.joiner_act, pred_init_state=getattr(m, "pred_init_state", None),
+                pred_init_out=getattr(m, "pred_init_out", None))
 
 
 NOALLOC_MAX_ROWS = 4096

@@ -17,6 +17,11 @@ __global__ void f32_to_bf16_kernel(const float* __restrict__ src, __nv_bfloat16*
   }
 }
 
+__global__ void bf16_to_f32_kernel(const __nv_bfloat16* __restrict__ src, float* __restrict__ dst, long long n) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) dst[i] = __bfloat162float(src[i]);
+}
+
 __global__ void gather_concat_bf16_kernel(const float* __restrict__ src1, const int* idx1, long long ld1, int K1,
                                           const float* __restrict__ src2, const int* idx2, long long ld2, int K2,
                                           const int* n_dev, int n_max, __nv_bfloat16* __restrict__ dst) {
@@ -135,6 +140,10 @@ void launch_f32_to_bf16(const float* src, __nv_bfloat16* dst, long long n, cudaS
   if (n <= 0) return;
   const long long threads = (n + 3) / 4;
   f32_to_bf16_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(src, dst, n);
+}
+
+void launch_bf16_to_f32(const __nv_bfloat16* src, float* dst, long long n, cudaStream_t st) {
+  if (n > 0) bf16_to_f32_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(src, dst, n);
 }
 
 void launch_gather_concat_bf16(const float* src1, const int* idx1, long long ld1, int K1, const float* src2,

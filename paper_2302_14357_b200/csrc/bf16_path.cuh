@@ -60,6 +60,7 @@ struct Bf16Mat {
 
 // elementwise helpers ---------------------------------------------------------------------------
 void launch_f32_to_bf16(const float* src, __nv_bfloat16* dst, long long n, cudaStream_t st);
+void launch_bf16_to_f32(const __nv_bfloat16* src, float* dst, long long n, cudaStream_t st);   // exact
 // dst[r, 0:K1] = src1 row (idx1 ? idx1[r] : r), dst[r, K1:K1+K2] = src2 row (idx2 ? idx2[r] : r)
 void launch_gather_concat_bf16(const float* src1, const int* idx1, long long ld1, int K1, const float* src2,
                                const int* idx2, long long ld2, int K2, const int* n_dev, int n_max,

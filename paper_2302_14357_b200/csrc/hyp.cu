@@ -521,7 +521,7 @@ __global__ void __launch_bounds__(1024) compact_kernel(HypState hs, int B, int T
       hs.row_slen[r] = hs.slen[b];
       if (hs.stateless) {
         const int ln = hs.slot_len[gs];
-        hs.row_p[r] = ln > 0 ? hs.slot_tok[gs * hs.U_cap + ln - 1] : hs.blank;
+        hs.row_p[r] = ln > 0 ? hs.slot_tok[gs * hs.U_cap + ln - 1] : hs.empty_row;
       } else {
         hs.row_p[r] = (int)gs;
       }

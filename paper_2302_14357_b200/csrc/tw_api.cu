@@ -32,10 +32,27 @@ int dev_alloc(tw_handle* h, T** p, size_t count) {
 
 #define TW_TRY(expr) do { int s_ = (expr); if (s_ != TW_OK) return s_; } while (0)
 
-int copy_weight(tw_handle* h, float** dst, const float* src, size_t count) {
+// float32 copy of a caller's tensor of the model's element type (bf16 -> float32 is exact)
+int copy_weight(tw_handle* h, float** dst, const void* src, size_t count) {
   TW_TRY(dev_alloc(h, dst, count));
-  TW_CUDA(h, cudaMemcpy(*dst, src, count * sizeof(float), cudaMemcpyDeviceToDevice));
+  if (h->dtype == TW_BF16) launch_bf16_to_f32(static_cast<const __nv_bfloat16*>(src), *dst, (long long)count, 0);
+  else TW_CUDA(h, cudaMemcpy(*dst, src, count * sizeof(float), cudaMemcpyDeviceToDevice));
   return TW_OK;
+}
+
+// Encoder frames of the caller's element type -> what the projection GEMM of this mode reads: the bf16 operand
+// buffer (TW_MODE_BF16) or float32 frames (TW_MODE_F32; the caller's own buffer when it is float32 already).
+const float* stage_frames(tw_handle* h, const void* enc, long long n, cudaStream_t st) {
+  if (h->mode == TW_MODE_BF16) {
+    if (h->dtype == TW_BF16) cudaMemcpyAsync(h->bf.enc.ptr, enc, (size_t)n * 2, cudaMemcpyDeviceToDevice, st);
+    else launch_f32_to_bf16(static_cast<const float*>(enc), h->bf.enc.ptr, n, st);
+    return nullptr;
+  }
+  if (h->dtype == TW_BF16) {
+    launch_bf16_to_f32(static_cast<const __nv_bfloat16*>(enc), h->enc_f32, n, st);
+    return h->enc_f32;
+  }
+  return static_cast<const float*>(enc);
 }
 
 // fp32 -> bf16 copy of a [rows, K] matrix with its tensor maps
@@ -144,13 +161,13 @@ void enqueue_predictor_slots(tw_handle* h, cudaStream_t st, int* launches, bool 
 }
 
 // E = enc W_e^T for `rows` frames
-void enqueue_project(tw_handle* h, const float* enc, int rows, float* E, cudaStream_t st, int* launches) {
+void enqueue_project(tw_handle* h, const void* enc, int rows, float* E, cudaStream_t st, int* launches) {
+  const float* enc32 = stage_frames(h, enc, (long long)rows * h->D_enc, st);
   if (h->mode == TW_MODE_BF16) {
-    launch_f32_to_bf16(enc, h->bf.enc.ptr, (long long)rows * h->D_enc, st);
     gemm_bf16(h, h->bf.enc, h->bf.W_e, nullptr, rows, E, nullptr, h->J, nullptr, st);
     *launches += 2;
   } else {
-    GemmOperand a{enc, nullptr, h->D_enc, h->W_e, h->D_enc, h->D_enc};
+    GemmOperand a{enc32, nullptr, h->D_enc, h->W_e, h->D_enc, h->D_enc};
     GemmOperand none{};
     GemmOut o{E, nullptr, h->J, nullptr};
     launch_gemm_f32(a, none, o, nullptr, rows, h->J, st);
@@ -271,6 +288,7 @@ int build_workspace(tw_handle* h) {
   hs.capSlot = N * (h->I_max + 1);
   hs.L = h->L; hs.Hd = h->Hd;
   hs.stateless = (h->pred_kind == TW_PRED_STATELESS);
+  hs.empty_row = h->blank;
   const size_t nb = (size_t)B, nslot = nb * hs.capSlot, nB = nb * hs.capB, R = (size_t)h->R_max;
   int** per_utt[] = {&hs.len, &hs.t0, &hs.slen, &hs.nA, &hs.nB, &hs.nTop, &hs.iters, &hs.status,
                      &hs.cursor, &hs.n_new, &hs.calls, &hs.joins, &hs.row_off, &hs.new_off, &hs.avail};
@@ -318,6 +336,7 @@ int build_workspace(tw_handle* h) {
   TW_TRY(dev_alloc(h, &hs.ldnb, R * h->V));
   TW_TRY(dev_alloc(h, &hs.logp, R * S * h->V));
   TW_TRY(dev_alloc(h, &h->E, (nb * h->max_T + 1) * h->J));   // + one dump row for frames a streamed chunk does not hold
+  if (h->mode == TW_MODE_F32 && h->dtype == TW_BF16) TW_TRY(dev_alloc(h, &h->enc_f32, nb * h->max_T * h->D_enc));
   TW_TRY(dev_alloc(h, &h->stream_oidx, nb * h->max_T));
   TW_TRY(dev_alloc(h, &h->zero_len, nb));
   TW_CUDA(h, cudaMemset(h->zero_len, 0, nb * sizeof(int)));
@@ -330,6 +349,7 @@ int build_workspace(tw_handle* h) {
 int init_impl(tw_handle* h, const tw_model* m, const tw_config* c) {
   h->D_enc = m->D_enc; h->P = m->P; h->J = m->J; h->V = m->V; h->blank = m->blank;
   h->pred_kind = m->pred_kind; h->emb_dim = m->emb_dim; h->joiner_act = m->joiner_act;
+  h->dtype = m->dtype; h->esize = m->dtype == TW_BF16 ? 2 : 4;
   h->L = (m->pred_kind == TW_PRED_LSTM) ? m->lstm_layers : 0;
   h->Hd = (m->pred_kind == TW_PRED_LSTM) ? m->lstm_hidden : 0;
   h->N = c->N; h->S = c->S; h->mode = c->mode; h->max_batch = c->max_batch; h->max_T = c->max_T;
@@ -352,25 +372,44 @@ int init_impl(tw_handle* h, const tw_model* m, const tw_config* c) {
   if (h->mode == TW_MODE_BF16) TW_TRY(build_bf16(h));
 
   int launches = 0;
+  GemmOperand none{};
+  float* init_out = nullptr;                 // InitPredictor's output as given by the caller (Sec. 3.2), float32
+  if (m->pred_init_out) TW_TRY(copy_weight(h, &init_out, m->pred_init_out, (size_t)h->P));
   if (h->pred_kind == TW_PRED_STATELESS) {
-    // W_p emb[k] for every token: the joiner rows index this table by their last token
-    TW_TRY(dev_alloc(h, &h->PpTab, (size_t)h->V * h->J));
+    // W_p emb[k] for every token: the joiner rows index this table by their last token.  A given initial output
+    // gets a row of its own after the vocabulary's, which serves the empty prefix.
+    TW_TRY(dev_alloc(h, &h->PpTab, (size_t)(h->V + 1) * h->J));
     GemmOperand a{h->emb, nullptr, h->emb_dim, h->W_p, h->P, h->P};
-    GemmOperand none{};
     GemmOut o{h->PpTab, nullptr, h->J, nullptr};
     launch_gemm_f32(a, none, o, nullptr, h->V, h->J, 0);
+    if (init_out) {
+      GemmOperand a1{init_out, nullptr, h->P, h->W_p, h->P, h->P};
+      GemmOut o1{h->PpTab + (size_t)h->V * h->J, nullptr, h->J, nullptr};
+      launch_gemm_f32(a1, none, o1, nullptr, 1, h->J, 0);
+      h->hs.empty_row = h->hs_fused.empty_row = h->V;
+    }
   } else {
-    // InitPredictor(): one step on the blank token from an all-zero state
     const size_t nhc = (size_t)h->L * 2 * h->Hd;
-    float* zero = nullptr; int* tok = nullptr;
-    TW_TRY(dev_alloc(h, &zero, nhc));
-    TW_TRY(dev_alloc(h, &tok, (size_t)1));
-    TW_TRY(dev_alloc(h, &h->init_hc, nhc));
     TW_TRY(dev_alloc(h, &h->init_Pp, (size_t)h->J));
-    TW_CUDA(h, cudaMemset(zero, 0, nhc * sizeof(float)));
-    TW_CUDA(h, cudaMemcpy(tok, &h->blank, sizeof(int), cudaMemcpyHostToDevice));
-    TW_TRY(enqueue_predictor_plain(h, tok, zero, 1, h->init_hc, h->init_Pp, 0, &launches));
-    h->hs.init_hc = h->init_hc; h->hs.init_Pp = h->init_Pp;
+    if (m->pred_init_state || init_out) {
+      // the caller's initial state; zeros without one; the output defaults to the top layer's h
+      if (m->pred_init_state) TW_TRY(copy_weight(h, &h->init_hc, m->pred_init_state, nhc));
+      else { TW_TRY(dev_alloc(h, &h->init_hc, nhc)); TW_CUDA(h, cudaMemset(h->init_hc, 0, nhc * sizeof(float))); }
+      const float* out = init_out ? init_out : h->init_hc + (size_t)(h->L - 1) * 2 * h->Hd;
+      GemmOperand a1{out, nullptr, h->P, h->W_p, h->P, h->P};
+      GemmOut o1{h->init_Pp, nullptr, h->J, nullptr};
+      launch_gemm_f32(a1, none, o1, nullptr, 1, h->J, 0);
+    } else {
+      // one step on the blank token from an all-zero state
+      float* zero = nullptr; int* tok = nullptr;
+      TW_TRY(dev_alloc(h, &zero, nhc));
+      TW_TRY(dev_alloc(h, &tok, (size_t)1));
+      TW_TRY(dev_alloc(h, &h->init_hc, nhc));
+      TW_CUDA(h, cudaMemset(zero, 0, nhc * sizeof(float)));
+      TW_CUDA(h, cudaMemcpy(tok, &h->blank, sizeof(int), cudaMemcpyHostToDevice));
+      TW_TRY(enqueue_predictor_plain(h, tok, zero, 1, h->init_hc, h->init_Pp, 0, &launches));
+    }
+    h->hs.init_hc = h->hs_fused.init_hc = h->init_hc; h->hs.init_Pp = h->hs_fused.init_Pp = h->init_Pp;
   }
   TW_CUDA(h, cudaGetLastError());
   TW_CUDA(h, cudaDeviceSynchronize());
@@ -459,6 +498,7 @@ int tw_init(const tw_model* m, const tw_config* c, tw_handle** out) {
   if (m->D_enc < 1 || m->P < 1 || m->J < 1 || m->V < 2 || m->emb_dim < 1) return TW_ERR_ARG;
   if (m->blank < 0 || m->blank >= m->V) return TW_ERR_ARG;
   if (m->joiner_act != TW_ACT_TANH && m->joiner_act != TW_ACT_RELU) return TW_ERR_ARG;
+  if (m->dtype != TW_F32 && m->dtype != TW_BF16) return TW_ERR_ARG;
   if (c->N < 1 || c->N > TW_MAX_BEAM || c->S < 1 || c->S > TW_MAX_SEGMENT) return TW_ERR_ARG;
   if (m->V - 1 < c->N) return TW_ERR_ARG;
   if (c->max_batch < 1 || c->max_T < 1 || c->max_iters_per_segment < 0 || c->max_tokens < 0) return TW_ERR_ARG;

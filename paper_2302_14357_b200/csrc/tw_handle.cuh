@@ -9,6 +9,9 @@ struct tw_handle {
   // model dimensions and search parameters
   int D_enc = 0, P = 0, J = 0, V = 0, blank = 0;
   int pred_kind = 0, emb_dim = 0, L = 0, Hd = 0, joiner_act = 0;
+  int dtype = 0;              // element type of the caller's weights and encoder frames (TW_F32 / TW_BF16)
+  size_t esize = 4;           // its size in bytes
+  float* enc_f32 = nullptr;   // TW_MODE_F32 with bf16 frames: their float32 copy [max_batch * max_T, D_enc]
   int N = 0, S = 0, mode = 0, max_batch = 0, max_T = 0, I_max = 0, U_cap = 0;
   int R_max = 0;
 
@@ -53,7 +56,7 @@ struct tw_handle {
   } bf;
 
   // staging of tw_decode_host (allocated on first use)
-  float* st_enc = nullptr; int* st_len = nullptr; int* st_tok = nullptr; int* st_lens = nullptr;
+  char* st_enc = nullptr; int* st_len = nullptr; int* st_tok = nullptr; int* st_lens = nullptr;
   // tw_decode_host uploads the frames in a few time chunks on copy_stream and decodes chunk k (as a streaming
   // session) while chunk k + 1 is still on its way
   static constexpr int kHostChunks = 3;

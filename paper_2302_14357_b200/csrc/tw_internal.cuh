@@ -140,6 +140,7 @@ struct HypState {
   int capSlot;   // hypothesis slots per utterance = N * (I_max + 1)
   int L, Hd;     // LSTM layers / hidden (0 for the stateless predictor)
   int stateless;
+  int empty_row;   // stateless predictor: row of the projected-output table that serves the empty token prefix
   // per utterance [B]
   int *len, *t0, *slen, *nA, *nB, *nTop, *iters, *status, *cursor, *n_new, *calls, *joins;
   int* avail;    // streaming: frames pushed so far (len is the part of them that may be decoded now)

@@ -7,7 +7,7 @@ from oracle import rnnt_model as rm
 
 def oracle_model(m: "tw_synth.SyntheticModel") -> rm.RnntModel:
     return rm.RnntModel(m.W_e, m.W_p, m.W_out, m.b_out, m.emb, m.lstm_W_ih, m.lstm_W_hh, m.lstm_b,
-                        activation=m.cfg.joiner_act)
+                        activation=m.cfg.joiner_act, pred_init_state=m.pred_init_state, pred_init_out=m.pred_init_out)
 
 
 def tiny_config(V=4, T=4, pred="stateless", seed=7, D_enc=5, J=6, emb=3, hidden=4, layers=1,

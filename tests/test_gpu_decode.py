@@ -70,6 +70,55 @@ def test_small_models_ragged_batch(pred, layers, S):
     _run(cfg, S, lengths=[0, 1, 23, 5, 17, 4])
 
 
+@pytest.mark.parametrize("pred,layers,what", [("lstm", 2, "state"), ("lstm", 1, "both"), ("lstm", 2, "out"), ("stateless", 0, "out")])
+def test_learned_initial_predictor_state(pred, layers, what):
+    """InitPredictor() as a caller-supplied quantity (Sec. 3.2): state and / or output of the empty prefix."""
+    cfg = _tiny(pred, layers, seed=13)
+    rng = np.random.default_rng(layers + len(what))
+
+    def mutate(m):
+        if what in ("state", "both"):
+            m.pred_init_state = (rng.standard_normal((layers, 2, cfg.lstm_hidden)) * 0.7).astype(np.float32)
+        if what in ("out", "both"):
+            m.pred_init_out = (rng.standard_normal(cfg.P) * 0.7).astype(np.float32)
+    _run(cfg, 3, lengths=[0, 1, 23, 5, 17, 4], mutate=mutate)
+    _run(cfg, 1, lengths=[3, 23, 2, 9, 1, 11], mutate=mutate)
+
+
+def test_bf16_weights_and_frames_at_the_boundary():
+    """tw_model::dtype = TW_BF16: weights and encoder frames cross the boundary as bfloat16.  On a bf16-representable
+    workload the decode is the float32-boundary decode bit for bit, in both arithmetic modes, from device frames,
+    from host frames (tw_decode_host) and as a streaming session."""
+    import torch
+    from paper_2302_14357_b200.binding import TwDecoder, weights_from_synth
+    cfg = tw_synth.WorkloadConfig("bd", 5, 50, (20, 50), 64, "lstm", 64, 2, 64, 128, 256, 3.0, 4, (3,), "bf16", 9)
+    m = tw_synth.make_model(cfg)
+    enc, lens = tw_synth.make_encoder_batch(cfg)
+    for mode in (0, 1):
+        a = TwDecoder(weights_from_synth(m), N=4, S=3, mode=mode, max_batch=5, max_T=50, dtype="f32")
+        b = TwDecoder(weights_from_synth(m), N=4, S=3, mode=mode, max_batch=5, max_T=50, dtype="bf16")
+        ref = [x.cpu().numpy() for x in a.decode(enc, lens)[:4]]
+        got = [x.cpu().numpy() for x in b.decode(torch.from_numpy(enc).to(torch.bfloat16).cuda(), lens)[:4]]
+        for x, y in zip(got, ref):
+            np.testing.assert_array_equal(x, y)
+        host = b.decode_host(torch.from_numpy(enc).to(torch.bfloat16).contiguous(), lens)[:4]
+        for x, y in zip(host, ref):
+            np.testing.assert_array_equal(x, y)
+        b.stream_open(5)
+        for t0 in range(0, 50, 20):
+            chunk = enc[:, t0:t0 + 20]
+            b.stream_push(chunk, np.clip(lens - t0, 0, chunk.shape[1]))
+        out = b.stream_close()
+        for x, y in zip(out[:4], ref):
+            np.testing.assert_array_equal(x.cpu().numpy(), y)
+        # the stage call takes frames of the handle's element type too
+        E_a = a.project_encoder(enc[0]).cpu().numpy()
+        E_b = b.project_encoder(torch.from_numpy(enc[0]).to(torch.bfloat16)).cpu().numpy()
+        np.testing.assert_array_equal(E_a, E_b)
+        a.close()
+        b.close()
+
+
 def test_iteration_cap_sets_limit_status():
     cfg = _tiny("stateless", V=12, seed=8).with_(blank_bias=-2.0)
     stats, _ = _run(cfg, 3, N=3, max_iters=2, lengths=[9, 9, 9, 9, 9, 9])

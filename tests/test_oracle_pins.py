@@ -155,6 +155,65 @@ def test_lstm_step_rows_matches_library_lstm_cell_batch(layers):
             np.testing.assert_allclose(c1[r, l], c[l], atol=1e-12)
 
 
+def test_learned_initial_predictor_state_lstm():
+    """InitPredictor() with a given state (Sec. 3.2).  (i) Giving the state that the default construction
+    reaches (one step on blank from zeros) changes nothing; (ii) the predictor outputs after a given state
+    follow torch.nn.LSTM started from that (h0, c0): a state that is ignored, or h and c exchanged, fails."""
+    torch = pytest.importorskip("torch")
+    cfg, model, enc = tiny_case(V=6, T=8, pred="lstm", seed=21, layers=2, blank_bias=1.5)
+    state, o = rm.predictor_init(model)
+    packed = np.stack([np.stack([state[0][l], state[1][l]]) for l in range(2)])        # [L, 2, Hd]
+    args = dict(W_e=model.W_e, W_p=model.W_p, W_out=model.W_out, b_out=model.b_out, emb=model.emb,
+                lstm_W_ih=model.lstm_W_ih, lstm_W_hh=model.lstm_W_hh, lstm_b=model.lstm_b)
+    same = rm.RnntModel(pred_init_state=packed, **args)
+    a, _ = tws.token_wise_beam_search(model, enc, 3, 2)
+    b, _ = tws.token_wise_beam_search(same, enc, 3, 2)
+    assert [t for t, _ in a] == [t for t, _ in b]
+    np.testing.assert_allclose([x for _, x in a], [x for _, x in b], atol=1e-12)
+    rng = np.random.default_rng(8)
+    Hd, E = model.lstm_W_hh[0].shape[1], model.emb.shape[1]
+    init = rng.standard_normal((2, 2, Hd))
+    learned = rm.RnntModel(pred_init_state=init, **args)
+    st0, o0 = rm.predictor_init(learned)
+    np.testing.assert_array_equal(o0, init[1, 0])                                      # the top layer's h
+    lib = torch.nn.LSTM(E, Hd, num_layers=2).double()
+    with torch.no_grad():
+        for l in range(2):
+            getattr(lib, f"weight_ih_l{l}").copy_(torch.from_numpy(model.lstm_W_ih[l]))
+            getattr(lib, f"weight_hh_l{l}").copy_(torch.from_numpy(model.lstm_W_hh[l]))
+            getattr(lib, f"bias_ih_l{l}").copy_(torch.from_numpy(model.lstm_b[l]))
+            getattr(lib, f"bias_hh_l{l}").zero_()
+        tokens = [3, 1, 5]
+        out, _ = lib(torch.from_numpy(model.emb[tokens]).unsqueeze(1),
+                     (torch.from_numpy(init[:, 0]).unsqueeze(1).contiguous(), torch.from_numpy(init[:, 1]).unsqueeze(1).contiguous()))
+    for i in range(len(tokens)):
+        _, oi = rm.predictor_for_tokens(learned, tokens[:i + 1])
+        np.testing.assert_allclose(oi, out[i, 0].numpy(), atol=1e-12)
+    # an explicit output overrides the top layer's h for the empty prefix only
+    both = rm.RnntModel(pred_init_state=init, pred_init_out=np.arange(Hd, dtype=float), **args)
+    _, ob = rm.predictor_init(both)
+    np.testing.assert_array_equal(ob, np.arange(Hd))
+    _, o1 = rm.predictor_for_tokens(both, [3])
+    np.testing.assert_allclose(o1, out[0, 0].numpy(), atol=1e-12)
+
+
+def test_learned_initial_predictor_output_stateless():
+    """Stateless predictor: the blank token is never a hypothesis's last token, so its embedding row serves only the
+    empty prefix; a given initial output must act exactly like a model whose blank row holds that vector."""
+    cfg, model, enc = tiny_case(V=6, T=8, pred="stateless", seed=22, blank_bias=1.5)
+    vec = np.linspace(-1.0, 1.0, model.emb.shape[1])
+    emb2 = model.emb.copy()
+    emb2[model.blank] = vec
+    swapped = rm.RnntModel(model.W_e, model.W_p, model.W_out, model.b_out, emb2)
+    given = rm.RnntModel(model.W_e, model.W_p, model.W_out, model.b_out, model.emb, pred_init_out=vec)
+    a, _ = tws.token_wise_beam_search(swapped, enc, 3, 2)
+    b, _ = tws.token_wise_beam_search(given, enc, 3, 2)
+    c, _ = tws.token_wise_beam_search(model, enc, 3, 2)
+    assert [t for t, _ in a] == [t for t, _ in b]
+    np.testing.assert_allclose([x for _, x in a], [x for _, x in b], atol=1e-12)
+    assert not np.allclose([x for _, x in b][:1], [x for _, x in c][:1], atol=1e-6)     # and it does change the search
+
+
 def test_stateless_predictor_is_embedding_of_last_token():
     emb = np.arange(12.0).reshape(4, 3)
     model = rm.RnntModel(np.zeros((2, 2)), np.zeros((2, 3)), np.zeros((4, 2)), np.zeros(4), emb)

@@ -49,7 +49,9 @@ class SyntheticModel:
     lstm_W_ih: List[np.ndarray] = field(default_factory=list)  # [4*Hd, in]
     lstm_W_hh: List[np.ndarray] = field(default_factory=list)  # [4*Hd, Hd]
     lstm_b: List[np.ndarray] = field(default_factory=list)     # [4*Hd]
-    pred_init: Optional[np.ndarray] = None
+    # a learned InitPredictor() result, when a test or a caller supplies one (the generators draw none)
+    pred_init_state: Optional[np.ndarray] = None   # [L, 2, Hd]
+    pred_init_out: Optional[np.ndarray] = None     # [P]
 
 
 def make_model(cfg: WorkloadConfig) -> SyntheticModel:
