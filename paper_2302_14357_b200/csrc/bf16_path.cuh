@@ -92,7 +92,8 @@ void launch_joiner_A_bf16(const JoinerRows& rows, __nv_bfloat16* A, cudaStream_t
 struct FusedJoinerParams {
   const int* R_dev; int R_max;       // hypothesis rows (device count optional)
   int S, V, K, blank, CL;            // CL = V / 256 CTAs per cluster; K = J
-  int no_max;                        // logits are bounded (|z| <= 40): softmax sums need no maximum
+  int no_max;                        // logits are bounded by zbound (at most 40): softmax sums need no maximum search
+  float zbound;                      // max_k (|W_out[k, :]|_1 + |b_out[k]|) >= |z| (tanh joiner); used when no_max
   const float* bias;                 // b_out [V]
   const float* ld_old;               // [R][S]
   const int* row_slen;               // [R] (nullptr: S)

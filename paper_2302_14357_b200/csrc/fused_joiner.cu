@@ -58,10 +58,11 @@ constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
 __device__ __forceinline__ float ex2f(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
 __device__ __forceinline__ float lg2f(float x) { float y; asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
 
-__device__ __forceinline__ float logaddexp_fast(float a, float b) {
+// log2(2^a + 2^b), branch-free; log 0 = -inf on either side or both
+__device__ __forceinline__ float logaddexp2_fast(float a, float b) {
   const float mx = fmaxf(a, b), mn = fminf(a, b);
-  if (mn == -INFINITY) return mx;
-  return mx + kLn2 * lg2f(1.f + ex2f((mn - mx) * kLog2e));
+  const float d = (mn == -INFINITY) ? -INFINITY : mn - mx;    // (-inf) - (-inf) would be NaN
+  return mx + lg2f(1.f + ex2f(d));
 }
 
 // sum over the S lanes [lane, lane + S) of x, valid in lanes whose window stays inside the warp.

@@ -340,16 +340,25 @@ __global__ void __launch_bounds__(2 * kStepThreads) hyp_step_kernel(HypState hs)
   __syncthreads();
   if (tid < kMaxBeam * kMaxBeam && s_ck[tid] >= 0) {
     const unsigned long long mine = s_key[tid];
-    int rank = 0;
-    // rows past H hold no candidate; an empty entry has the key of log 0, which ranks below every candidate
-    // (candidates are finite), so it needs no validity test
+    const int h = tid / kMaxBeam, jj = tid % kMaxBeam;
+    // Rank = how many candidates come before this one in the order (score desc, h asc, k asc).  Every row's list is
+    // sorted that way and padded with the key of log 0, so the candidates of a row that come before this one are a
+    // prefix of its list: its length is found by bisection (four probes and a last one for a full list) instead of
+    // a look at all sixteen entries.  Rows before h count their ties with this score, rows after it do not, and in
+    // its own row exactly the jj entries ahead of it count.
+    int rank = jj;
     for (int hh = 0; hh < H; ++hh) {
+      if (hh == h) continue;
+      const unsigned long long* key = s_key + hh * kMaxBeam;
+      const bool ties = hh < h;
+      int cnt = 0;
 #pragma unroll
-      for (int j = 0; j < kMaxBeam; ++j) {
-        const int o = hh * kMaxBeam + j;
-        const unsigned long long so = s_key[o];
-        rank += (so > mine || (so == mine && o < tid)) ? 1 : 0;
+      for (int st = kMaxBeam / 2; st > 0; st >>= 1) {
+        const unsigned long long so = key[cnt + st - 1];
+        if (so > mine || (ties && so == mine)) cnt += st;
       }
+      if (cnt == kMaxBeam - 1) { const unsigned long long so = key[cnt]; cnt += (so > mine || (ties && so == mine)) ? 1 : 0; }
+      rank += cnt;
     }
     if (rank < N) s_sel[rank] = tid;
   }

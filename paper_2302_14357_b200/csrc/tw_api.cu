@@ -245,6 +245,7 @@ int build_bf16(tw_handle* h) {
       launch_logit_bound(h->bf.W_out.ptr, h->b_out, h->V, h->J, bound_dev, 0);
       TW_CUDA(h, cudaMemcpy(&bound, bound_dev, sizeof(float), cudaMemcpyDeviceToHost));
       h->bf.no_max = (bound <= 40.f) && h->joiner_act == TW_ACT_TANH;   // the bound needs |act| <= 1
+      h->bf.zbound = bound;
       TW_TRY(make_bf16_mat(h, &h->bf.A_tiled, nullptr, fused_joiner_A_rows(h->R_max, h->S), h->J, true, false));
       TW_TRY(dev_alloc(h, &h->bf.lse, (size_t)h->R_max * h->S));
       TW_TRY(scan_select_setup());
@@ -460,7 +461,7 @@ int enqueue_joiner_fused(tw_handle* h, const JoinerRows& rows, const float* ld_o
   if (ldnb == nullptr) ldnb = h->bf.ldnb_pad;   // a caller's buffer has V columns: only with an unpadded vocabulary
   FusedJoinerParams fp{};
   fp.R_dev = rows.R_dev; fp.R_max = rows.R_max; fp.S = rows.S; fp.V = h->bf.Vp; fp.K = rows.J; fp.blank = h->blank;
-  fp.CL = h->bf.CL; fp.no_max = h->bf.no_max ? 1 : 0; fp.bias = h->bf.bias_pad; fp.ld_old = ld_old; fp.row_slen = rows.row_slen;
+  fp.CL = h->bf.CL; fp.no_max = h->bf.no_max ? 1 : 0; fp.zbound = h->bf.zbound; fp.bias = h->bf.bias_pad; fp.ld_old = ld_old; fp.row_slen = rows.row_slen;
   fp.ldphi = ldphi; fp.la = la; fp.lse = h->bf.lse; fp.ldnb = ldnb; fp.err = h->bf.err; fp.clear_word = clear_word;
   TW_TRY(launch_fused_joiner(h->bf.A_tiled.as_A, h->bf.W_out_pad.as_B256, fp, h->bf.max_clusters, st));
   if (mark_fn) mark_fn(h, 2, st);       // the fused kernel alone

@@ -43,6 +43,7 @@ struct tw_handle {
     int* err = nullptr;                                   // device error word of the bounded waits
     // fused joiner + softmax + Eq. 3-7 + selection (logits stay in tensor memory)
     bool fused_ok = false, fused_on = false, no_max = false;
+    float zbound = 0.f;                                   // bound of |logit| behind no_max
     int CL = 0, max_clusters = 0;
     // The fused kernel splits the vocabulary into 256-column CTAs.  A vocabulary that is not a multiple of 256 is
     // padded for it: Vp columns, the added rows of W_out zero and their bias -1e30 (probability 0, never a
