@@ -10,8 +10,9 @@ import numpy as np
 from . import rnnt_model as rm
 
 
-def _lattice_log_probs(model: rm.RnntModel, enc: np.ndarray, y: Sequence[int]) -> np.ndarray:
-    """log J(t, u, .) for every frame t and every prefix length u of y: [T, U+1, V]."""
+def _lattice_log_probs(model: rm.RnntModel, enc: np.ndarray, y: Sequence[int], blank_threshold=None) -> np.ndarray:
+    """log J(t, u, .) for every frame t and every prefix length u of y: [T, U+1, V].  With a blank threshold the
+    lattice nodes whose blank probability exceeds it keep their blank arc only."""
     outs = []
     state, o = rm.predictor_init(model)
     outs.append(o)
@@ -19,13 +20,15 @@ def _lattice_log_probs(model: rm.RnntModel, enc: np.ndarray, y: Sequence[int]) -
         state, o = rm.predictor_step(model, state, k)
         outs.append(o)
     logJ = rm.joiner_log_probs(model, np.asarray(enc, dtype=np.float64), np.stack(outs))  # [U+1, T, V]
+    if blank_threshold is not None:
+        logJ, _ = rm.apply_blank_threshold(logJ, blank_threshold, model.blank)
     return np.transpose(logJ, (1, 0, 2))
 
 
-def forward_log_prob(model: rm.RnntModel, enc: np.ndarray, y: Sequence[int]) -> float:
+def forward_log_prob(model: rm.RnntModel, enc: np.ndarray, y: Sequence[int], blank_threshold=None) -> float:
     """alpha(t, u) = alpha(t-1, u) J(t-1, u, blank) + alpha(t, u-1) J(t, u-1, y_u);
     p(y|x) = alpha(T-1, U) J(T-1, U, blank)   (0-based frames)."""
-    lj = _lattice_log_probs(model, enc, y)
+    lj = _lattice_log_probs(model, enc, y, blank_threshold)
     T, U = lj.shape[0], len(y)
     blank = model.blank
     alpha = np.full((T, U + 1), -np.inf)
@@ -40,11 +43,11 @@ def forward_log_prob(model: rm.RnntModel, enc: np.ndarray, y: Sequence[int]) -> 
     return float(alpha[T - 1, U] + lj[T - 1, U, blank])
 
 
-def brute_force_log_prob(model: rm.RnntModel, enc: np.ndarray, y: Sequence[int]) -> float:
+def brute_force_log_prob(model: rm.RnntModel, enc: np.ndarray, y: Sequence[int], blank_threshold=None) -> float:
     """Sum, in the linear domain, over every monotone alignment: from (t, u) a
     blank moves to (t+1, u), token y_{u+1} moves to (t, u+1); an alignment is
     complete when the blank of the last frame has been taken with u = U."""
-    lj = _lattice_log_probs(model, enc, y)
+    lj = _lattice_log_probs(model, enc, y, blank_threshold)
     J = np.exp(lj)
     T, U = J.shape[0], len(y)
     blank = model.blank
@@ -78,7 +81,7 @@ def forward_log_prob_monotonic(model: rm.RnntModel, enc: np.ndarray, y: Sequence
 
 def brute_force_log_prob_monotonic(model: rm.RnntModel, enc: np.ndarray, y: Sequence[int]) -> float:
     """Sum over every way to place the U tokens on distinct frames, in order; all other frames emit blank."""
-    lj = _lattice_log_probs(model, enc, y)
+    lj = _lattice_log_probs(model, enc, y, blank_threshold)
     J = np.exp(lj)
     T, U = J.shape[0], len(y)
     blank = model.blank

@@ -22,7 +22,7 @@ class RnntModel:
     def __init__(self, W_e, W_p, W_out, b_out, emb,
                  lstm_W_ih: Sequence = (), lstm_W_hh: Sequence = (), lstm_b: Sequence = (),
                  blank: int = 0, activation: str = "tanh",
-                 pred_init_state=None, pred_init_out=None):
+                 pred_init_state=None, pred_init_out=None, normalisation: str = "softmax"):
         self.W_e = _f64(W_e)        # [J, D_enc]
         self.W_p = _f64(W_p)        # [J, P]
         self.W_out = _f64(W_out)    # [V, J]
@@ -34,6 +34,11 @@ class RnntModel:
         self.blank = int(blank)
         assert activation in ("tanh", "relu")
         self.activation = activation
+        # "softmax": J = softmax over the whole vocabulary (Sec. 3.1).  "hat": the factorised output that blank
+        # thresholding needs (Sec. 2, Sec. 5): the blank logit goes through a sigmoid of its own and the
+        # remaining probability is shared out by a softmax over the non-blank tokens.
+        assert normalisation in ("softmax", "hat")
+        self.normalisation = normalisation
         # InitPredictor() of Sec. 3.2 returns a learned initial state: optional here, as
         # pred_init_state [L, 2, Hd] (per layer h then c) and / or pred_init_out [P]
         self.pred_init_state = None if pred_init_state is None else _f64(pred_init_state)
@@ -64,7 +69,48 @@ def joiner_log_probs(model: RnntModel, seg: np.ndarray, pred_out: np.ndarray) ->
     pre = e[None, :, :] + p[:, None, :]             # [H, S', J]
     hidden = np.tanh(pre) if model.activation == "tanh" else np.maximum(pre, 0.0)
     z = hidden @ model.W_out.T + model.b_out        # [H, S', V]
+    if model.normalisation == "hat":
+        return log_hat(z, model.blank)
     return log_softmax(z)
+
+
+def log_hat(z: np.ndarray, blank: int = 0) -> np.ndarray:
+    """Factorised output distribution over the last axis, in log space:
+      p(blank) = sigmoid(z_blank),   p(k) = (1 - p(blank)) * exp(z_k) / sum_{k' != blank} exp(z_k')   for k != blank."""
+    zb = z[..., blank]
+    log_pb = -np.logaddexp(0.0, -zb)                # log sigmoid(zb)
+    log_rest = -np.logaddexp(0.0, zb)               # log (1 - sigmoid(zb))
+    lab = np.delete(z, blank, axis=-1)
+    m = lab.max(axis=-1, keepdims=True)
+    lse = (m + np.log(np.exp(lab - m).sum(axis=-1, keepdims=True)))[..., 0]
+    out = z - lse[..., None] + log_rest[..., None]
+    out[..., blank] = log_pb
+    return out
+
+
+def apply_blank_threshold(logJ: np.ndarray, threshold: float, blank: int = 0, flip=None) -> np.ndarray:
+    """Blank thresholding (Sec. 2: above a threshold on the blank probability the joiner is not invoked; Sec. 5
+    names it as a later extension and prints no equations, so the rule here is this code's reading): at every
+    (.., frame) whose blank probability exceeds `threshold` the label part of the output is not computed, i.e.
+    the non-blank entries become probability 0 while the blank probability stays what the blank head gave.
+    threshold = 1 changes nothing.  logJ [..., V] -> (thresholded copy, boolean mask of the skipped positions).
+    `flip`, if given, is called with |log p(blank) - log threshold| per position (row-major order) and returns True
+    where that decision is to be inverted."""
+    lb = logJ[..., blank]
+    with np.errstate(divide="ignore"):
+        lt = np.log(threshold)
+    skip = lb > lt
+    if flip is not None:
+        flat = skip.reshape(-1)
+        for i, gap in enumerate(np.abs(lb - lt).reshape(-1)):
+            if flip(float(gap)):
+                flat[i] = not flat[i]
+        skip = flat.reshape(skip.shape)
+    out = logJ.copy()
+    keep_blank = out[..., blank].copy()
+    out[skip] = -np.inf
+    out[..., blank] = keep_blank
+    return out, skip
 
 
 def _sigmoid(x):

@@ -75,6 +75,8 @@ class SearchStats:
     frames: int = 0
     calls: int = 0               # joiner invocations (Calls/Frame numerator)
     joins: int = 0               # frames fed to the joiner (Joins/Frame numerator)
+    frame_rows: int = 0          # (hypothesis, frame) pairs fed to the joiner
+    skipped: int = 0             # of those, pairs whose label part blank thresholding left out
     limit_hit: bool = False
     iters_per_segment: List[int] = field(default_factory=list)
 
@@ -130,12 +132,16 @@ def token_wise_beam_search(model: rm.RnntModel, enc: np.ndarray, N: int, S: int,
                            max_iters: Optional[int] = None,
                            max_len: Optional[int] = None,
                            log: Optional[DecisionLog] = None,
-                           monotonic: bool = False):
+                           monotonic: bool = False,
+                           blank_threshold: Optional[float] = None):
     """Algorithm 1.  enc [T, D_enc] -> (list of (tokens, log score) best first, stats).
 
     max_iters: safety cap on inner-loop passes per segment (None = uncapped).
     max_len:   test-only cap on hypothesis length; longer expansions are never
-               created (used to make the un-pruned search finite)."""
+               created (used to make the un-pruned search finite).
+    blank_threshold: blank thresholding for a model with the factorised output (rnnt_model.apply_blank_threshold):
+               (hypothesis, frame) pairs whose blank probability exceeds it contribute their blank
+               probability only; stats.skipped counts them.  None or 1: plain Algorithm 1."""
     enc = np.asarray(enc, dtype=np.float64)
     T = enc.shape[0]
     blank = model.blank
@@ -164,6 +170,11 @@ def token_wise_beam_search(model: rm.RnntModel, enc: np.ndarray, N: int, S: int,
             logJ = rm.joiner_log_probs(model, seg, pred)          # [H, S', V]
             stats.calls += 1
             stats.joins += Sp
+            stats.frame_rows += Sp * len(A)
+            if blank_threshold is not None:
+                flip = (lambda gap: log.decide("skip", gap)) if log is not None else None
+                logJ, skipped = rm.apply_blank_threshold(logJ, blank_threshold, blank, flip)
+                stats.skipped += int(skipped.sum())
 
             ld_old = np.stack([hyp.ld for hyp in A])              # [H, S']
             lBl = sm.blank_product(logJ, blank)                   # Eq. 3

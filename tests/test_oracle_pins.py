@@ -556,3 +556,102 @@ def test_monotonic_pruned_scores_never_exceed_exact_probability(S):
     for y, s in nbest:
         assert s <= ef.forward_log_prob_monotonic(model, enc, y) + 1e-10
     assert max(stats.iters_per_segment) <= S + 1     # at most one token per frame, then everything has left
+
+
+# ---- blank thresholding on a factorised output (Sec. 2, Sec. 5; the rule is this build's reading) ----------------
+def _hat_case(**kw):
+    cfg, model, enc = tiny_case(**kw)
+    hat = rm.RnntModel(model.W_e, model.W_p, model.W_out, model.b_out, model.emb, model.lstm_W_ih, model.lstm_W_hh,
+                       model.lstm_b, normalisation="hat")
+    return cfg, hat, enc
+
+
+def test_hat_output_hand_worked_golden():
+    rows = _read_golden("hat_closed_form.txt")
+    z1 = np.array([np.log(3.0), 0.0, np.log(2.0)])
+    z2 = np.array([np.log(2.0), -np.log(4.0), 0.0])
+    np.testing.assert_allclose(np.exp(rm.log_hat(z1[None], 0))[0], rows[0], atol=1e-12)
+    np.testing.assert_allclose(np.exp(rm.log_hat(z2[None], 1))[0], rows[1], atol=1e-12)
+    # through the joiner: a distribution per (hypothesis, frame), blank probability = sigmoid of the blank logit
+    cfg, hat, enc = _hat_case(V=6, T=5, pred="lstm", seed=3)
+    _, o = rm.predictor_init(hat)
+    lj = rm.joiner_log_probs(hat, enc, o[None])
+    np.testing.assert_allclose(np.exp(lj).sum(axis=-1), 1.0, atol=1e-12)
+    soft = rm.RnntModel(hat.W_e, hat.W_p, hat.W_out, hat.b_out, hat.emb, hat.lstm_W_ih, hat.lstm_W_hh, hat.lstm_b)
+    ls = rm.joiner_log_probs(soft, enc, o[None])
+    # same logits underneath: ratios between non-blank tokens are those of the plain softmax
+    np.testing.assert_allclose(lj[..., 2] - lj[..., 3], ls[..., 2] - ls[..., 3], atol=1e-12)
+    # and the blank probability is the logistic function of the blank logit itself
+    z0 = np.tanh(enc @ hat.W_e.T + o @ hat.W_p.T) @ hat.W_out[0] + hat.b_out[0]
+    np.testing.assert_allclose(np.exp(lj[0, :, 0]), 1.0 / (1.0 + np.exp(-z0)), atol=1e-12)
+
+
+def test_blank_threshold_rule_on_a_table():
+    logJ = np.log(np.array([[[0.7, 0.2, 0.1], [0.4, 0.5, 0.1]], [[0.95, 0.03, 0.02], [0.6, 0.3, 0.1]]]))
+    out, skip = rm.apply_blank_threshold(logJ, 0.65, 0)
+    assert skip.tolist() == [[True, False], [True, False]]
+    np.testing.assert_allclose(np.exp(out[0, 0]), [0.7, 0.0, 0.0], atol=1e-15)
+    np.testing.assert_allclose(np.exp(out[0, 1]), [0.4, 0.5, 0.1], atol=1e-15)
+    np.testing.assert_allclose(np.exp(out[1, 0]), [0.95, 0.0, 0.0], atol=1e-15)
+    same, none = rm.apply_blank_threshold(logJ, 1.0, 0)
+    assert not none.any() and np.array_equal(same, logJ)
+    allb, every = rm.apply_blank_threshold(logJ, 0.0, 0)
+    assert every.all() and np.all(np.isneginf(allb[..., 1:])) and np.array_equal(allb[..., 0], logJ[..., 0])
+
+
+@pytest.mark.parametrize("pred", ["stateless", "lstm"])
+@pytest.mark.parametrize("T,S,tau", [(4, 1, 1.0), (4, 2, 1.0), (4, 3, 0.5), (5, 2, 0.35), (4, 4, 0.6), (6, 4, 0.45), (3, 50, 0.5)])
+def test_unpruned_search_with_blank_threshold_is_exact(pred, T, S, tau):
+    """Nothing pruned: every sequence gets exactly the sum over its alignments on the thresholded lattice (nodes
+    whose blank probability exceeds the threshold keep their blank arc only), for every segment size.  tau = 1 is
+    plain Algorithm 1 on the factorised distribution."""
+    V, U = 4, 2 if T > 4 else 3
+    cfg, hat, enc = _hat_case(V=V, T=T, pred=pred, seed=T * 10 + S, blank_bias=0.0)
+    seqs = list(_all_sequences(V, U))
+    nbest, stats = tws.token_wise_beam_search(hat, enc, N=10 * len(seqs), S=S, max_len=U, blank_threshold=tau)
+    got = dict(nbest)
+    assert stats.skipped == 0 or tau < 1.0
+    for y in seqs:
+        with np.errstate(divide="ignore"):
+            fwd = ef.forward_log_prob(hat, enc, y, blank_threshold=tau)
+            brute = ef.brute_force_log_prob(hat, enc, y, blank_threshold=tau) if T <= 5 else fwd
+        if np.isneginf(fwd):
+            assert y not in got or np.isneginf(got[y])
+            continue
+        assert got[y] == pytest.approx(fwd, abs=1e-11)
+        assert brute == pytest.approx(fwd, abs=1e-11)
+    assert stats.frame_rows >= stats.joins and stats.skipped <= stats.frame_rows
+
+
+def test_blank_threshold_zero_keeps_only_the_empty_hypothesis():
+    """Threshold 0: every frame is skipped, no token is ever emitted, and the score is the product of the blank
+    probabilities of the empty prefix along the utterance."""
+    cfg, hat, enc = _hat_case(V=6, T=9, pred="lstm", seed=12)
+    nbest, stats = tws.token_wise_beam_search(hat, enc, 3, 4, blank_threshold=0.0)
+    _, o = rm.predictor_init(hat)
+    lj = rm.joiner_log_probs(hat, enc, o[None])[0]
+    assert [t for t, _ in nbest] == [()]
+    assert nbest[0][1] == pytest.approx(lj[:, 0].sum(), abs=1e-12)
+    assert stats.skipped == stats.frame_rows == 9 and stats.calls == 3
+
+
+def test_blank_threshold_mass_accounting():
+    """delta_phi + sum_k delta_nb + (mass of the label parts left out) = sum_t d_old, with the left-out mass written
+    as the explicit sum over the skipped frames t2 of sum_{t1 <= t2} d_old(t1) Bl(t1, t2) (1 - J(t2, blank))."""
+    rng = np.random.default_rng(5)
+    H, S, V = 3, 4, 7
+    logJ = rm.log_hat(rng.standard_normal((H, S, V)) * 2.0, 0)
+    ld_old = rng.standard_normal((H, S)) - 1.0
+    thr, skip = rm.apply_blank_threshold(logJ, 0.4, 0)
+    assert skip.any() and not skip.all()
+    lBl = sm.blank_product(thr)
+    ld = sm.nonblank_expansion_t(thr, lBl, ld_old)
+    nb = np.exp(sm.nonblank_expansion(ld))[:, 1:].sum(axis=1)
+    phi = np.exp(sm.blank_expansion(lBl, ld_old))
+    left_out = np.zeros(H)
+    for h in range(H):
+        for t2 in range(1, S + 1):
+            if skip[h, t2 - 1]:
+                a = sum(np.exp(ld_old[h, t1 - 1] + lBl[h, t1, t2]) for t1 in range(1, t2 + 1))
+                left_out[h] += a * (1.0 - np.exp(logJ[h, t2 - 1, 0]))
+    np.testing.assert_allclose(phi + nb + left_out, np.exp(ld_old).sum(axis=1), rtol=1e-12)
