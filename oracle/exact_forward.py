@@ -81,7 +81,7 @@ def forward_log_prob_monotonic(model: rm.RnntModel, enc: np.ndarray, y: Sequence
 
 def brute_force_log_prob_monotonic(model: rm.RnntModel, enc: np.ndarray, y: Sequence[int]) -> float:
     """Sum over every way to place the U tokens on distinct frames, in order; all other frames emit blank."""
-    lj = _lattice_log_probs(model, enc, y, blank_threshold)
+    lj = _lattice_log_probs(model, enc, y)
     J = np.exp(lj)
     T, U = J.shape[0], len(y)
     blank = model.blank
