@@ -42,6 +42,9 @@ def parse_args():
     ap.add_argument("--no-fused", action="store_true", help="bf16 mode: staged joiner kernels instead of the fused one")
     ap.add_argument("--monotonic", action="store_true", help="the monotonic RNN-T variant (every output consumes a frame)")
     ap.add_argument("--cpu-frames", type=int, default=0, help="frames of the CPU-baseline sample (0: auto)")
+    ap.add_argument("--blank-threshold", type=float, default=None,
+                    help="blank thresholding for a workload with the factorised output (h1): skip the label part of a "
+                         "(hypothesis, frame) whose blank probability exceeds this")
     ap.add_argument("--no-largest", action="store_true", help="skip the fused kernel's leg at the largest step shape")
     ap.add_argument("--agreement-utterances", type=int, default=4, help="utterances of the bf16 top-1 agreement check (0: skip)")
     return ap.parse_args()
@@ -97,7 +100,7 @@ def measured_peaks():
 
 # ------------------------------------------------------------------------------------------------
 # CPU baseline: the oracle as it stands, on a bounded sample of the same workload
-def oracle_sample(cfg, S, frames, utt=0, monotonic=False):
+def oracle_sample(cfg, S, frames, utt=0, monotonic=False, blank_threshold=None):
     from oracle import rnnt_model as rm
     from oracle import token_wise_search as tws
     try:
@@ -108,10 +111,11 @@ def oracle_sample(cfg, S, frames, utt=0, monotonic=False):
     m = tw_synth.make_model(cfg)
     enc, lens = tw_synth.make_encoder_batch(cfg, batch=utt + 1)
     om = rm.RnntModel(m.W_e, m.W_p, m.W_out, m.b_out, m.emb, m.lstm_W_ih, m.lstm_W_hh, m.lstm_b,
-                      activation=cfg.joiner_act)
+                      activation=cfg.joiner_act, normalisation=cfg.joiner_norm)
     n = int(min(frames, lens[utt]))
     t0 = time.perf_counter()
-    _, st = tws.token_wise_beam_search(om, enc[utt, :n], cfg.N, S, max_iters=4 * S + 16, monotonic=monotonic)
+    _, st = tws.token_wise_beam_search(om, enc[utt, :n], cfg.N, S, max_iters=4 * S + 16, monotonic=monotonic,
+                                       blank_threshold=blank_threshold)
     dt = time.perf_counter() - t0
     return {"value": n / dt, "unit": UNIT, "cores": int(cores), "kind": "oracle",
             "sample": "utterance %d of workload %s, first %d frames, N=%d S=%d, fp64 numpy; %.1f s"
@@ -119,7 +123,7 @@ def oracle_sample(cfg, S, frames, utt=0, monotonic=False):
             "calls_per_frame": st.calls / max(n, 1), "joins_per_frame": st.joins / max(n, 1)}, dt
 
 
-def top1_agreement(dec, cfg, S, enc_np, len_np, utterances, frames, monotonic=False):
+def top1_agreement(dec, cfg, S, enc_np, len_np, utterances, frames, monotonic=False, blank_threshold=None):
     """bf16 mode against the fp64 oracle: both decode the first `frames` frames of a few utterances of the
     bench batch; reports how often the best token sequence is the same and the largest score gap where it is."""
     from oracle import rnnt_model as rm
@@ -132,10 +136,11 @@ def top1_agreement(dec, cfg, S, enc_np, len_np, utterances, frames, monotonic=Fa
     tokens, olens, scores = tokens.cpu().numpy(), olens.cpu().numpy(), scores.cpu().numpy()
     m = tw_synth.make_model(cfg)
     om = rm.RnntModel(m.W_e, m.W_p, m.W_out, m.b_out, m.emb, m.lstm_W_ih, m.lstm_W_hh, m.lstm_b,
-                      activation=cfg.joiner_act)
+                      activation=cfg.joiner_act, normalisation=cfg.joiner_norm)
     agree, gap = 0, 0.0
     for b in range(K):
-        ref, _ = tws.token_wise_beam_search(om, enc[b, :lens[b]], cfg.N, S, max_iters=4 * S + 16, monotonic=monotonic)
+        ref, _ = tws.token_wise_beam_search(om, enc[b, :lens[b]], cfg.N, S, max_iters=4 * S + 16, monotonic=monotonic,
+                                            blank_threshold=blank_threshold)
         got = tuple(int(x) for x in tokens[b, 0, :max(int(olens[b, 0]), 0)])
         if got == ref[0][0]:
             agree += 1
@@ -195,10 +200,10 @@ def run_reference(args, cfg, S):
         return
     frames = args.cpu_frames or max(12, auto_cpu_frames(cfg) // 4)
     for _ in range(args.warmup):
-        oracle_sample(cfg, S, max(4, frames // 4), monotonic=args.monotonic)
+        oracle_sample(cfg, S, max(4, frames // 4), monotonic=args.monotonic, blank_threshold=args.blank_threshold)
     times, vals, last = [], [], None
     for k in range(args.steps):
-        last, dt = oracle_sample(cfg, S, frames, utt=0, monotonic=args.monotonic)
+        last, dt = oracle_sample(cfg, S, frames, utt=0, monotonic=args.monotonic, blank_threshold=args.blank_threshold)
         times.append(dt)
         vals.append(last["value"])
     value = frames * len(times) / sum(times) if times else 0.0
@@ -291,6 +296,8 @@ def run_ours(args, cfg, S):
         dec.set_lanes(False)
     if args.monotonic:
         dec.set_monotonic(True)
+    if args.blank_threshold is not None and dec.set_blank_threshold(args.blank_threshold) != 0:
+        raise RuntimeError("--blank-threshold needs a workload with the factorised output (h1) and a value in [0, 1]")
     enc = torch.from_numpy(enc_np).cuda()
     lens = torch.from_numpy(len_np).cuda()
     frames = int(len_np.sum())
@@ -385,12 +392,13 @@ def run_ours(args, cfg, S):
         "ms_per_step": ms / args.steps, "ms_per_step_with_stage_events": ms_profiled / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": mode_name, "data": "synthetic",
         "config": {"workload": cfg.name, "B_per_gpu": B, "T": cfg.T, "N": cfg.N, "S": S, "J": cfg.J, "V": cfg.V,
-                   "mode": mode_name, "variant": "monotonic" if args.monotonic else "standard", "l2": ("inputs larger than L2 (encoder batch %.0f MB)" % (enc_np.nbytes / 1e6)) if flush is None
+                   "mode": mode_name, "variant": "monotonic" if args.monotonic else "standard", "joiner_norm": cfg.joiner_norm,
+                   "blank_threshold": args.blank_threshold, "l2": ("inputs larger than L2 (encoder batch %.0f MB)" % (enc_np.nbytes / 1e6)) if flush is None
                          else "L2 flushed by a 256 MB write before every timed step (encoder batch %.0f MB)" % (enc_np.nbytes / 1e6),
                    "parallelism": "independent utterance batches per GPU, no collective"},
         "calls_per_frame": st["calls"] / max(st["frames"], 1), "joins_per_frame": st["joins"] / max(st["frames"], 1),
         "device_steps_per_decode": st["steps"], "avg_rows_per_step": st["rows"] / max(st["steps"], 1),
-        "limit_hits": st["limit_hits"],
+        "limit_hits": st["limit_hits"], "frame_rows_skipped_share": st["frame_rows_skipped"] / max(st["joiner_frame_rows"], 1),
         "stage_share": {k[3:]: round(v / tot_ns, 4) for k, v in stage_ns.items()},
         "stage_ms_per_decode": {k[3:]: round(v * 1e-6, 3) for k, v in stage_ns.items()},
         "roofline": {"kernel": joiner_kernel_name(mode_name, st), "bound": "tensor", "achieved": achieved, "peak": peak,
@@ -415,9 +423,10 @@ def run_ours(args, cfg, S):
             line["roofline_largest"] = big
     if mode_name == "bf16" and world == 1 and not args.no_cpu_baseline and args.agreement_utterances > 0:
         line["bf16_top1_agreement"] = top1_agreement(dec, cfg, S, enc_np, len_np, args.agreement_utterances,
-                                                     min(150, args.cpu_frames or auto_cpu_frames(cfg)), args.monotonic)
+                                                     min(150, args.cpu_frames or auto_cpu_frames(cfg)), args.monotonic, args.blank_threshold)
     if not args.no_cpu_baseline and world == 1:
-        line["cpu_baseline"], _ = oracle_sample(cfg, S, args.cpu_frames or auto_cpu_frames(cfg), monotonic=args.monotonic)
+        line["cpu_baseline"], _ = oracle_sample(cfg, S, args.cpu_frames or auto_cpu_frames(cfg), monotonic=args.monotonic,
+                                                 blank_threshold=args.blank_threshold)
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

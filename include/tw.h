@@ -47,6 +47,7 @@ enum { TW_MODE_F32 = 0, TW_MODE_BF16 = 1 };   /* arithmetic of the decoder (tw_c
 enum { TW_F32 = 0, TW_BF16 = 1 };             /* element type of the caller's weights and frames (tw_model::dtype) */
 enum { TW_PRED_STATELESS = 0, TW_PRED_LSTM = 1 };
 enum { TW_ACT_TANH = 0, TW_ACT_RELU = 1 };   /* joiner hidden nonlinearity */
+enum { TW_NORM_SOFTMAX = 0, TW_NORM_HAT = 1 }; /* how the joiner's logits become probabilities (tw_model::joiner_norm) */
 
 #define TW_MAX_BEAM 16     /* N <= 16 */
 #define TW_MAX_SEGMENT 64  /* S <= 64 */
@@ -78,6 +79,9 @@ typedef struct {
   int32_t pred_kind, emb_dim, lstm_layers, lstm_hidden;
   int32_t joiner_act; /* TW_ACT_TANH or TW_ACT_RELU */
   int32_t dtype;      /* TW_F32 or TW_BF16 */
+  int32_t joiner_norm; /* TW_NORM_SOFTMAX: J = softmax(z) (Sec. 3.1).  TW_NORM_HAT: the factorised output that blank
+                          thresholding needs (Sec. 2): p(blank) = sigmoid(z_blank), and p(k) = (1 - p(blank)) *
+                          softmax over the non-blank tokens; row `blank` of W_out is then the blank head */
   const void* W_e;   /* [J, D_enc] */
   const void* W_p;   /* [J, P]     */
   const void* W_out; /* [V, J]     */
@@ -124,6 +128,7 @@ typedef struct {
   int64_t joiner_launches; /* launches summed in ns_joiner                             */
   int64_t fused_clusters;  /* clusters the fused joiner keeps resident (0: fused path unavailable) */
   int64_t fused_on;        /* 1 if tw_decode takes the fused joiner path                          */
+  int64_t frame_rows_skipped; /* of joiner_frame_rows, the (row, frame) pairs blank thresholding left out */
 } tw_stats;
 
 /* Builds a decoder: copies (and in bf16 mode converts) the weights, runs InitPredictor, allocates
@@ -305,6 +310,16 @@ int tw_set_lanes(tw_handle* h, int on);
  * tw_set_inline_gather(h, 0) leaves both to a kernel of their own (one more launch per step, a work list in a fixed
  * order).  Both give the same N-best.  TW_ERR_STATE if the handle has no such path, or while a streaming session is open. */
 int tw_set_inline_gather(tw_handle* h, int on);
+
+/* Blank thresholding (Sec. 2 and Sec. 5 name it as a way to skip joiner work that adds to the gains of Algorithm 1;
+ * the paper prints no equations for it).  Only for a TW_NORM_HAT model, whose blank probability comes from a head of
+ * its own.  A (hypothesis, frame) pair whose blank probability exceeds `threshold` contributes that blank probability
+ * only: its non-blank terms drop out of Eq. 4-6.  threshold = 1 (the default) skips nothing, threshold = 0 skips every
+ * pair.  tw_stats::frame_rows_skipped counts the skipped pairs of a decode.  TW_MODE_F32 and the staged TW_MODE_BF16
+ * kernels drop the terms after the contraction; the fused kernel masks them in its epilogue (its tile layout keeps a
+ * lane per frame, so the contraction's row count does not shrink).  TW_ERR_STATE for a softmax model or while a
+ * streaming session is open, TW_ERR_ARG for a threshold outside [0, 1]. */
+int tw_set_blank_threshold(tw_handle* h, float threshold);
 
 /* Monotonic RNN-T variant (Sec. 2 and Sec. 5 name it as an adjustment of Algorithm 1; the paper prints no
  * equations for it).  Every output, blank or token, consumes one frame, so at most one token is emitted

@@ -9,11 +9,12 @@ MODE_F32, MODE_BF16 = 0, 1
 PRED_STATELESS, PRED_LSTM = 0, 1
 ACT_TANH, ACT_RELU = 0, 1
 DT_F32, DT_BF16 = 0, 1
+NORM_SOFTMAX, NORM_HAT = 0, 1
 TW_OK, TW_ERR_ARG, TW_ERR_ALLOC, TW_ERR_CUDA, TW_ERR_LIMIT, TW_ERR_STATE, TW_ERR_TIMEOUT = range(7)
 
 EXPORTED_SYMBOLS = [
     "tw_init", "tw_destroy", "tw_decode", "tw_decode_host", "tw_max_tokens", "tw_project_encoder",
-    "tw_joiner_segment", "tw_expand", "tw_joiner_expand", "tw_predictor_step", "tw_get_stats", "tw_set_profiling", "tw_set_fused", "tw_set_graph", "tw_set_lanes", "tw_set_monotonic", "tw_set_inline_gather",
+    "tw_joiner_segment", "tw_expand", "tw_joiner_expand", "tw_predictor_step", "tw_get_stats", "tw_set_profiling", "tw_set_fused", "tw_set_graph", "tw_set_lanes", "tw_set_monotonic", "tw_set_inline_gather", "tw_set_blank_threshold",
     "tw_stream_open", "tw_stream_push", "tw_stream_nbest", "tw_stream_close",
     "tw_joiner_expand_noalloc",
     "tw_last_cuda_error", "tw_strerror",
@@ -31,7 +32,7 @@ class TwError(RuntimeError):
 
 
 class _Model(C.Structure):
-    _fields_ = [(n, C.c_int32) for n in ("D_enc", "P", "J", "V", "blank", "pred_kind", "emb_dim", "lstm_layers", "lstm_hidden", "joiner_act", "dtype")] + \
+    _fields_ = [(n, C.c_int32) for n in ("D_enc", "P", "J", "V", "blank", "pred_kind", "emb_dim", "lstm_layers", "lstm_hidden", "joiner_act", "dtype", "joiner_norm")] + \
                [(n, C.c_void_p) for n in ("W_e", "W_p", "W_out", "b_out", "emb", "host_lstm_W_ih", "host_lstm_W_hh", "host_lstm_b",
                                           "pred_init_state", "pred_init_out")]
 
@@ -42,7 +43,8 @@ class _Config(C.Structure):
 
 class _Stats(C.Structure):
     _fields_ = [(n, C.c_int64) for n in ("frames", "calls", "joins", "steps", "rows", "kernel_launches", "limit_hits", "joiner_frame_rows",
-                                          "ns_prologue", "ns_predictor", "ns_joiner", "ns_scan", "ns_hyp", "joiner_launches", "fused_clusters", "fused_on")]
+                                          "ns_prologue", "ns_predictor", "ns_joiner", "ns_scan", "ns_hyp", "joiner_launches", "fused_clusters", "fused_on",
+                                          "frame_rows_skipped")]
 
 
 def lib_path() -> str:
@@ -77,6 +79,7 @@ def load_library() -> C.CDLL:
     lib.tw_set_lanes.argtypes = [vp, C.c_int]
     lib.tw_set_monotonic.argtypes = [vp, C.c_int]
     lib.tw_set_inline_gather.argtypes = [vp, C.c_int]
+    lib.tw_set_blank_threshold.argtypes = [vp, C.c_float]
     lib.tw_stream_open.argtypes = [vp, i32, vp]
     lib.tw_stream_push.argtypes = [vp, vp, vp, i32, vp]
     lib.tw_stream_nbest.argtypes = [vp, vp, vp, vp, vp, vp]
@@ -111,7 +114,7 @@ class TwDecoder:
 
     def __init__(self, weights: Dict, N: int, S: int, mode: int = MODE_F32, max_batch: int = 1, max_T: int = 1,
                  max_iters_per_segment: int = 0, max_tokens: int = 0, blank: int = 0, joiner_act: str = "tanh",
-                 dtype: str = "f32"):
+                 dtype: str = "f32", joiner_norm: str = "softmax"):
         import torch
         self._torch = torch
         self.lib = load_library()
@@ -127,6 +130,7 @@ class TwDecoder:
             return t.to(self.device).to(self._tdtype).contiguous()
         weights = dict(weights)
         joiner_act = weights.pop("joiner_act", None) or joiner_act
+        joiner_norm = weights.pop("joiner_norm", None) or joiner_norm
         w = {k: ([dev(a) for a in v] if isinstance(v, (list, tuple)) else dev(v)) for k, v in weights.items() if v is not None}
         self._keep = w
         layers = len(w.get("lstm_W_ih", []))
@@ -141,6 +145,7 @@ class TwDecoder:
         m.lstm_hidden = w["lstm_W_hh"][0].shape[1] if layers else 0
         m.joiner_act = {"tanh": ACT_TANH, "relu": ACT_RELU}[joiner_act]
         m.dtype = {"f32": DT_F32, "bf16": DT_BF16}[dtype]
+        m.joiner_norm = {"softmax": NORM_SOFTMAX, "hat": NORM_HAT}[joiner_norm]
         for name in ("pred_init_state", "pred_init_out"):
             setattr(m, name, w[name].data_ptr() if name in w else None)
         for name in ("W_e", "W_p", "W_out", "b_out", "emb"):
@@ -324,6 +329,10 @@ class TwDecoder:
         """tw_set_inline_gather: who builds the predictor's work list in a fused bf16 decode step."""
         self._check(self.lib.tw_set_inline_gather(self.h, int(bool(on))), "tw_set_inline_gather")
 
+    def set_blank_threshold(self, threshold: float) -> int:
+        """tw_set_blank_threshold (factorised-output models only); returns the status."""
+        return self.lib.tw_set_blank_threshold(self.h, float(threshold))
+
     def set_lanes(self, on: bool):
         self._check(self.lib.tw_set_lanes(self.h, int(bool(on))), "tw_set_lanes")
 
@@ -340,7 +349,7 @@ def weights_from_synth(m) -> Dict:
     """tw_model fields from a tw_synth.SyntheticModel (plain attribute access, no arithmetic)."""
     return dict(W_e=m.W_e, W_p=m.W_p, W_out=m.W_out, b_out=m.b_out, emb=m.emb,
                 lstm_W_ih=list(m.lstm_W_ih), lstm_W_hh=list(m.lstm_W_hh), lstm_b=list(m.lstm_b),
-                joiner_act=m.cfg.joiner_act, pred_init_state=getattr(m, "pred_init_state", None),
+                joiner_act=m.cfg.joiner_act, joiner_norm=getattr(m.cfg, "joiner_norm", "softmax"), pred_init_state=getattr(m, "pred_init_state", None),
                 pred_init_out=getattr(m, "pred_init_out", None))
 
 

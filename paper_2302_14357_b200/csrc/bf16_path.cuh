@@ -100,6 +100,9 @@ struct FusedJoinerParams {
   float* ldphi; float* la; float* lse;   // [R], [R][S], [R][S]
   float* ldnb;                       // [R][V] delta_nb as a probability ratio, NOT its log (0 at the blank column)
   int* err;
+  int hat;                           // factorised output (JoinerRows::hat); log2_tau = log2 of the blank threshold
+  float log2_tau;
+  unsigned long long* skipped;       // optional counter of the (row, frame) pairs blank thresholding left out
   int* clear_word;                   // optional: one device word the kernel sets to 0 once its predecessors have finished
 };
 bool fused_joiner_eligible(int S, int V, int J);

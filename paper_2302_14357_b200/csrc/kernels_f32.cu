@@ -167,8 +167,9 @@ __global__ void __launch_bounds__(256) log_softmax_kernel(JoinerRows jr, int bla
     for (int k = tid; k < jr.V; k += 256) row[k] = (k == blank) ? 0.f : -INFINITY;
     return;
   }
+  const bool hat = jr.hat != 0;
   float mx = -INFINITY;
-  for (int k = tid; k < jr.V; k += 256) mx = fmaxf(mx, row[k]);
+  for (int k = tid; k < jr.V; k += 256) if (!hat || k != blank) mx = fmaxf(mx, row[k]);
   mx = warp_max(mx);
   if (lane == 0) red[w] = mx;
   __syncthreads();
@@ -176,7 +177,7 @@ __global__ void __launch_bounds__(256) log_softmax_kernel(JoinerRows jr, int bla
   __syncthreads();
   mx = bcast;
   float s = 0.f;
-  for (int k = tid; k < jr.V; k += 256) s += expf(row[k] - mx);
+  for (int k = tid; k < jr.V; k += 256) if (!hat || k != blank) s += expf(row[k] - mx);
   s = warp_sum(s);
   __syncthreads();
   if (lane == 0) red[w] = s;
@@ -184,7 +185,19 @@ __global__ void __launch_bounds__(256) log_softmax_kernel(JoinerRows jr, int bla
   if (tid == 0) { float v = 0.f; for (int i = 0; i < 8; ++i) v += red[i]; bcast = mx + logf(v); }
   __syncthreads();
   const float lse = bcast;
-  for (int k = tid; k < jr.V; k += 256) row[k] = row[k] - lse;
+  if (!hat) {
+    for (int k = tid; k < jr.V; k += 256) row[k] = row[k] - lse;
+    return;
+  }
+  // factorised output: log sigmoid(zb), log(1 - sigmoid(zb)) without cancellation
+  const float zb = row[blank];
+  __syncthreads();                               // every thread has read the blank logit before it is overwritten
+  const float sp = (zb >= 0.f) ? log1pf(expf(-zb)) : -zb + log1pf(expf(zb));     // softplus(-zb)
+  const float log_pb = -sp, log_rest = -sp - zb;
+  const bool skip = log_pb > jr.log_tau;         // blank thresholding: the label part is left out
+  if (skip && tid == 0 && jr.skipped != nullptr) atomicAdd(jr.skipped, 1ull);
+  for (int k = tid; k < jr.V; k += 256)
+    row[k] = (k == blank) ? log_pb : (skip ? -INFINITY : row[k] - lse + log_rest);
 }
 
 // One CTA per hypothesis row.  Eq. 3-7 through the occupancy recursion

@@ -3,6 +3,7 @@
 #include <vector>
 #include <stdio.h>
 #include <string.h>
+#include <math.h>
 
 #include "tw_handle.cuh"
 
@@ -322,7 +323,7 @@ int build_workspace(tw_handle* h) {
   for (int** p : per_row) TW_TRY(dev_alloc(h, p, R));
   TW_TRY(dev_alloc(h, &hs.row_ld, R * S));
   TW_TRY(dev_alloc(h, &hs.scalars, (size_t)kScCount));
-  TW_TRY(dev_alloc(h, &hs.rows_total, (size_t)2));
+  TW_TRY(dev_alloc(h, &hs.rows_total, (size_t)3));
   TW_TRY(dev_alloc(h, &hs.ldphi, R));
   TW_TRY(dev_alloc(h, &hs.la, R * S));
   if (scan_select_fits(S, h->V)) {
@@ -342,7 +343,7 @@ int build_workspace(tw_handle* h) {
   TW_TRY(dev_alloc(h, &h->zero_len, nb));
   TW_CUDA(h, cudaMemset(h->zero_len, 0, nb * sizeof(int)));
   TW_CUDA(h, cudaMemset(hs.scalars, 0, kScCount * sizeof(int)));
-  TW_CUDA(h, cudaMemset(hs.rows_total, 0, 2 * sizeof(long long)));
+  TW_CUDA(h, cudaMemset(hs.rows_total, 0, 3 * sizeof(long long)));
   TW_CUDA(h, cudaHostAlloc((void**)&h->host_flag, (kScCount + 4) * sizeof(long long), cudaHostAllocDefault));
   return TW_OK;
 }
@@ -351,6 +352,7 @@ int init_impl(tw_handle* h, const tw_model* m, const tw_config* c) {
   h->D_enc = m->D_enc; h->P = m->P; h->J = m->J; h->V = m->V; h->blank = m->blank;
   h->pred_kind = m->pred_kind; h->emb_dim = m->emb_dim; h->joiner_act = m->joiner_act;
   h->dtype = m->dtype; h->esize = m->dtype == TW_BF16 ? 2 : 4;
+  h->hat = m->joiner_norm == TW_NORM_HAT ? 1 : 0;
   h->L = (m->pred_kind == TW_PRED_LSTM) ? m->lstm_layers : 0;
   h->Hd = (m->pred_kind == TW_PRED_LSTM) ? m->lstm_hidden : 0;
   h->N = c->N; h->S = c->S; h->mode = c->mode; h->max_batch = c->max_batch; h->max_T = c->max_T;
@@ -435,13 +437,13 @@ void enqueue_joiner_expand_f32(tw_handle* h, const JoinerRows& rows, const float
 void enqueue_scan(tw_handle* h, const JoinerRows& rows, const float* ld_old, float* logp, float* ldphi,
                   float* ldnb, float* la, double* ldphi_d, double* la_d, const CandOut& cand, cudaStream_t st,
                   int* launches) {
-  if (h->hs.lse != nullptr) {
+  if (h->hs.lse != nullptr && !h->hat) {
     ScanSelectArgs a{logp, ld_old, rows.row_slen, rows.R_dev, rows.R_max, rows.S, rows.V, h->blank,
                      h->hs.lse, ldphi, ldnb, la, ldphi_d, la_d, cand};
     launch_scan_select(a, h->mode == TW_MODE_BF16, st);
     *launches += 1;
   } else {
-    launch_log_softmax(rows, h->blank, logp, st);
+    launch_log_softmax(rows, h->blank, logp, st);        // factorised output and blank thresholding included (rows.hat)
     launch_expand_f32(logp, ld_old, rows.row_slen, rows.R_dev, rows.R_max, rows.S, rows.V, h->blank, ldphi,
                       ldnb, la, ldphi_d, la_d, cand, st);
     *launches += 2;
@@ -463,6 +465,7 @@ int enqueue_joiner_fused(tw_handle* h, const JoinerRows& rows, const float* ld_o
   fp.R_dev = rows.R_dev; fp.R_max = rows.R_max; fp.S = rows.S; fp.V = h->bf.Vp; fp.K = rows.J; fp.blank = h->blank;
   fp.CL = h->bf.CL; fp.no_max = h->bf.no_max ? 1 : 0; fp.zbound = h->bf.zbound; fp.bias = h->bf.bias_pad; fp.ld_old = ld_old; fp.row_slen = rows.row_slen;
   fp.ldphi = ldphi; fp.la = la; fp.lse = h->bf.lse; fp.ldnb = ldnb; fp.err = h->bf.err; fp.clear_word = clear_word;
+  fp.hat = rows.hat; fp.log2_tau = rows.log_tau * 1.4426950408889634f; fp.skipped = rows.skipped;
   TW_TRY(launch_fused_joiner(h->bf.A_tiled.as_A, h->bf.W_out_pad.as_B256, fp, h->bf.max_clusters, st));
   if (mark_fn) mark_fn(h, 2, st);       // the fused kernel alone
   *launches += 2;
@@ -500,6 +503,7 @@ int tw_init(const tw_model* m, const tw_config* c, tw_handle** out) {
   if (m->blank < 0 || m->blank >= m->V) return TW_ERR_ARG;
   if (m->joiner_act != TW_ACT_TANH && m->joiner_act != TW_ACT_RELU) return TW_ERR_ARG;
   if (m->dtype != TW_F32 && m->dtype != TW_BF16) return TW_ERR_ARG;
+  if (m->joiner_norm != TW_NORM_SOFTMAX && m->joiner_norm != TW_NORM_HAT) return TW_ERR_ARG;
   if (c->N < 1 || c->N > TW_MAX_BEAM || c->S < 1 || c->S > TW_MAX_SEGMENT) return TW_ERR_ARG;
   if (m->V - 1 < c->N) return TW_ERR_ARG;
   if (c->max_batch < 1 || c->max_T < 1 || c->max_iters_per_segment < 0 || c->max_tokens < 0) return TW_ERR_ARG;
@@ -592,6 +596,19 @@ int tw_set_inline_gather(tw_handle* h, int on) {
     const bool can = x->mode == TW_MODE_BF16 && x->bf.fused_ok && x->hs_fused.defer_rows && x->pred_kind != TW_PRED_STATELESS;
     if (on && !can) return TW_ERR_STATE;
     if (can) x->hs_fused.inline_gather = on ? 1 : 0;
+    if (x->graph_exec) { cudaGraphExecDestroy(x->graph_exec); x->graph_exec = nullptr; }   // captured arguments are by value
+  }
+  return TW_OK;
+}
+
+int tw_set_blank_threshold(tw_handle* h, float threshold) {
+  if (!h) return TW_ERR_ARG;
+  if (!(threshold >= 0.f && threshold <= 1.f)) return TW_ERR_ARG;
+  if (!h->hat || h->stream_B > 0) return TW_ERR_STATE;
+  tw_handle* all[3] = {h, h->lane[0], h->lane[1]};
+  for (tw_handle* x : all) {
+    if (!x) continue;
+    x->log_tau = threshold > 0.f ? logf(threshold) : -INFINITY;
     if (x->graph_exec) { cudaGraphExecDestroy(x->graph_exec); x->graph_exec = nullptr; }   // captured arguments are by value
   }
   return TW_OK;

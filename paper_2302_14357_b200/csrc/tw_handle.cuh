@@ -9,6 +9,8 @@ struct tw_handle {
   // model dimensions and search parameters
   int D_enc = 0, P = 0, J = 0, V = 0, blank = 0;
   int pred_kind = 0, emb_dim = 0, L = 0, Hd = 0, joiner_act = 0;
+  int hat = 0;                // TW_NORM_HAT model: factorised output
+  float log_tau = 0.f;        // log of the blank threshold (0: nothing is skipped)
   int dtype = 0;              // element type of the caller's weights and encoder frames (TW_F32 / TW_BF16)
   size_t esize = 4;           // its size in bytes
   float* enc_f32 = nullptr;   // TW_MODE_F32 with bf16 frames: their float32 copy [max_batch * max_T, D_enc]

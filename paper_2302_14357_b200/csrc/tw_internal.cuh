@@ -93,6 +93,12 @@ struct JoinerRows {
   const int* R_dev;      // device row count (nullptr: use R_max)
   int R_max, S, J, V;
   int act;               // TW_ACT_TANH / TW_ACT_RELU
+  // Factorised output (TW_NORM_HAT): p(blank) = sigmoid(z_blank), the rest shared out by a softmax over the other
+  // tokens; a (row, frame) with log p(blank) > log_tau keeps its blank probability only (blank thresholding) and
+  // is counted in *skipped.  hat == 0: plain softmax, the two other fields are not read.
+  int hat = 0;
+  float log_tau = 0.f;
+  unsigned long long* skipped = nullptr;
 };
 // z[(r,t), k] = sum_j tanh(E[e0[r]+t, j] + Pp[p[r], j]) * W_out[k, j] + b_out[k]; rows of padding
 // frames (t >= slen) are left untouched.

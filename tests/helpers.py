@@ -7,7 +7,8 @@ from oracle import rnnt_model as rm
 
 def oracle_model(m: "tw_synth.SyntheticModel") -> rm.RnntModel:
     return rm.RnntModel(m.W_e, m.W_p, m.W_out, m.b_out, m.emb, m.lstm_W_ih, m.lstm_W_hh, m.lstm_b,
-                        activation=m.cfg.joiner_act, pred_init_state=m.pred_init_state, pred_init_out=m.pred_init_out)
+                        activation=m.cfg.joiner_act, pred_init_state=m.pred_init_state, pred_init_out=m.pred_init_out,
+                        normalisation=getattr(m.cfg, "joiner_norm", "softmax"))
 
 
 def tiny_config(V=4, T=4, pred="stateless", seed=7, D_enc=5, J=6, emb=3, hidden=4, layers=1,
@@ -52,21 +53,23 @@ def _same_nbest(ref, got, tol, tau):
     return True
 
 
-def check_against_oracle(model, enc, N, S, max_iters, got, tol=SCORE_TOL, tau=TIE_TAU, max_flips=6, monotonic=False):
+def check_against_oracle(model, enc, N, S, max_iters, got, tol=SCORE_TOL, tau=TIE_TAU, max_flips=6, monotonic=False,
+                         blank_threshold=None):
     """Runs Algorithm 1 in the oracle and compares with `got`.  Returns (ok, how, stats) where how is
     'exact' or 'near-tie' (the oracle reproduces `got` after inverting one or two pruning decisions
     whose score gap is below tau)."""
     import itertools
     from oracle import token_wise_search as tws
     log = tws.DecisionLog()
-    ref, stats = tws.token_wise_beam_search(model, enc, N, S, max_iters=max_iters, log=log, monotonic=monotonic)
+    ref, stats = tws.token_wise_beam_search(model, enc, N, S, max_iters=max_iters, log=log, monotonic=monotonic,
+                                            blank_threshold=blank_threshold)
     if _same_nbest(ref, got, tol, tau):
         return True, "exact", stats
     close = log.below(tau)[:max_flips]
     for n in (1, 2):
         for flips in itertools.combinations(close, n):
             ref2, _ = tws.token_wise_beam_search(model, enc, N, S, max_iters=max_iters, log=tws.DecisionLog(flips),
-                                                 monotonic=monotonic)
+                                                 monotonic=monotonic, blank_threshold=blank_threshold)
             if _same_nbest(ref2, got, tol, tau):
                 return True, "near-tie", stats
     return False, "mismatch: oracle %r vs %r (min margin %.3g)" % (ref[:2], got[:2], log.min_margin()), stats

@@ -23,6 +23,7 @@ class WorkloadConfig:
     dtype: str                  # "f32" | "bf16": storage precision of weights/inputs
     seed: int
     joiner_act: str = "tanh"   # "tanh" | "relu"
+    joiner_norm: str = "softmax"   # "softmax" | "hat": factorised output, row 0 of W_out is the blank head
 
     @property
     def P(self) -> int:
@@ -53,6 +54,10 @@ CONFIGS = {
     # 3-layer LSTM predictor; the vocabulary is not a multiple of anything
     "p1": WorkloadConfig("p1", 32, 300, (150, 300), 512, "lstm", 512, 3, 512,
                          512, 501, 4.0, 5, (1, 3, 5), "bf16", 3, "relu"),
+    # the Librispeech-shaped model with a factorised (HAT) output for blank thresholding (Sec. 2, Sec. 5): the blank
+    # head's bias makes the blank probability about 0.8 on most (hypothesis, frame) pairs
+    "h1": WorkloadConfig("h1", 64, 400, (400, 400), 512, "lstm", 640, 1, 640,
+                         640, 1024, 1.5, 10, (3,), "bf16", 4, "tanh", "hat"),
 }
 
 
