@@ -114,7 +114,9 @@ void launch_logit_bound(const __nv_bfloat16* W, const float* bias, int V, int J,
 // dst[r, k] = log src[r * ld_src + k] (log 0 = -inf) for r < R, k < V; dst rows have V columns (dst may be src when
 // ld_src == V)
 void launch_log_rows(const float* src, long long ld_src, float* dst, int R, int V, cudaStream_t st);
-void launch_joiner_A_tiled(const JoinerRows& rows, __nv_bfloat16* A, cudaStream_t st);
+// pf_base / pf_bytes (optional): a constant matrix the kernel asks into L2 for its successor (16-byte aligned)
+void launch_joiner_A_tiled(const JoinerRows& rows, __nv_bfloat16* A, cudaStream_t st, const void* pf_base = nullptr,
+                           long long pf_bytes = 0);
 // the same for the rows of a decode step (utterance b's rows are row_off[b] .. + nA[b] - 1, all on one segment)
 void launch_joiner_A_tiled_utt(const JoinerRows& rows, const int* row_off, const int* nA, int B, __nv_bfloat16* A,
                                cudaStream_t st);

@@ -262,13 +262,19 @@ constexpr uint32_t kWideABytes = BM * BK * 2, kWideBBytes = kWideMaxBN * BK * 2;
 constexpr size_t kWideSmem = (size_t)kWideStages * (kWideABytes + kWideBBytes) + 1024 + 256;
 
 // The LSTM cell on one CTA's accumulator tile: rows m0 .. m0 + 127, gate columns n0 .. n0 + 32 nu - 1 (TMEM columns
-// 0 .. 32 nu - 1).  Called by the 16 epilogue warps (warp = 2 .. 17) once acc_full has been armed.
-__device__ __forceinline__ void lstm_tile_epilogue(const GemmBf16Params& p, uint32_t tmem_base, uint64_t* acc_full, int M,
-                                                   int m0, int n0, int nu, int warp, int lane) {
-  // Epilogue: the LSTM cell, a row per thread; warp group grp takes the 32-column chunks grp, grp + 4, grp + 8.
+// 0 .. 32 nu - 1).  Called by the 16 epilogue warps (warp = 2 .. 17).  Two things keep the part after the contraction
+// short.  (1) What is added to the products - the bias, or layer 0's table row W_ih emb[token] + b - is written into
+// tensor memory BEFORE the contraction, which then accumulates onto it from its first instruction: the gather of
+// those rows (128 bytes per thread and chunk, scattered) runs while the first operand tiles are still on their way,
+// and the MMA thread waits on acc_init for it.  (2) The parents' cell states of all of a warp's chunks are fetched
+// into registers during the contraction.  After it a chunk is one tensor-memory load, the cell and three stores.
+constexpr int kWideMaxChunks = (kWideMaxBN / 32 + 3) / 4;      // chunks of 32 columns a warp can own (groups of 4 warps)
+__device__ __forceinline__ void lstm_tile_epilogue(const GemmBf16Params& p, uint32_t tmem_base, uint64_t* acc_full,
+                                                   uint64_t* acc_init, int M, int m0, int n0, int nu, int warp, int lane) {
+  // a row per thread; warp group grp takes the 32-column chunks grp, grp + 4, grp + 8
   const int ew = warp - 2, q = warp & 3, grp = ew >> 2;
   const int m = m0 + q * 32 + lane;
-  const bool live = m < M;                                   // tcgen05.ld below is warp-wide: idle rows stay in the loop
+  const bool live = m < M;                                   // tcgen05 accesses below are warp-wide: idle rows stay in the loops
   const long long stride = (long long)p.lstm.L * 2 * p.lstm.Hd, lo = (long long)p.lstm.l * 2 * p.lstm.Hd;
   const float* cin = nullptr;
   const float* arow = nullptr;
@@ -279,60 +285,82 @@ __device__ __forceinline__ void lstm_tile_epilogue(const GemmBf16Params& p, uint
     hout = p.lstm.hc_out + (long long)(p.lstm.idx_out ? p.lstm.idx_out[m] : m) * stride + lo;
     xrow = p.lstm.xnext + (long long)m * p.lstm.ld_xnext;
     if (p.addend) arow = p.addend + (long long)(p.add_idx ? p.add_idx[m] : m) * p.ld_add;
-    // while the contraction runs: pull this thread's epilogue inputs (table row segments, parent's c) into L2
-    for (int c = grp; c < nu; c += kWideEpiWarps / 4) {
-      if (arow) prefetch_l2(arow + n0 + c * 32);
-      prefetch_l2(cin + ((n0 + c * 32) >> 2));
-    }
   }
   // 256-bit accesses when every row segment this kernel touches starts on a 32-byte boundary
   const bool wide_ok = (p.lstm.Hd & 7) == 0 &&
                        ((reinterpret_cast<uintptr_t>(p.lstm.hc_in) | reinterpret_cast<uintptr_t>(p.lstm.hc_out) |
                          reinterpret_cast<uintptr_t>(p.addend) | (uintptr_t)(p.ld_add * 4)) & 31) == 0;
+  const uint32_t tlane = tmem_base + ((uint32_t)(q * 32) << 16);
+  // ---- (1) the accumulators start as bias + addend
+#pragma unroll 1
+  for (int c = grp; c < nu; c += kWideEpiWarps / 4) {
+    float v[32];
+    const int nb = n0 + c * 32;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] = 0.f;
+    if (p.bias) {
+#pragma unroll
+      for (int j = 0; j < 32; j += 4) {
+        const float4 b4 = __ldg(reinterpret_cast<const float4*>(p.bias + nb + j));
+        v[j] = b4.x; v[j + 1] = b4.y; v[j + 2] = b4.z; v[j + 3] = b4.w;
+      }
+    }
+    if (arow) {
+      if (wide_ok) {
+#pragma unroll
+        for (int j = 0; j < 32; j += 8) {
+          float a8[8];
+          ld_global_v8(arow + nb + j, a8);
+#pragma unroll
+          for (int u = 0; u < 8; ++u) v[j + u] += a8[u];
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < 32; j += 4) {
+          const float4 a4 = __ldg(reinterpret_cast<const float4*>(arow + nb + j));
+          v[j] += a4.x; v[j + 1] += a4.y; v[j + 2] += a4.z; v[j + 3] += a4.w;
+        }
+      }
+    }
+    tmem_st32(tlane + (uint32_t)(c * 32), v);
+  }
+  tmem_st_wait();
+  tc_fence_before();
+  __syncwarp();
+  if (lane == 0) mbar_arrive(acc_init);
+  // ---- (2) the parents' cell states, while the contraction runs
+  float cp[kWideMaxChunks][8];
+#pragma unroll
+  for (int i = 0; i < kWideMaxChunks; ++i) {
+    const int c = grp + i * (kWideEpiWarps / 4);
+#pragma unroll
+    for (int u = 0; u < 8; ++u) cp[i][u] = 0.f;
+    if (live && c < nu) {
+      const int j0 = (n0 + c * 32) >> 2;                       // 8 whole hidden units (gate columns interleaved)
+      if (wide_ok) {
+        ld_global_v8(cin + j0, cp[i]);
+      } else {
+        const float4 c0 = *reinterpret_cast<const float4*>(cin + j0), c1 = *reinterpret_cast<const float4*>(cin + j0 + 4);
+        cp[i][0] = c0.x; cp[i][1] = c0.y; cp[i][2] = c0.z; cp[i][3] = c0.w; cp[i][4] = c1.x; cp[i][5] = c1.y; cp[i][6] = c1.z; cp[i][7] = c1.w;
+      }
+    }
+  }
   bool ok = mbar_wait(acc_full, 0, p.err);
   ok = __all_sync(0xffffffffu, ok);
   if (ok) {
     tc_fence_after();
-#pragma unroll 1
-    for (int c = grp; c < nu; c += kWideEpiWarps / 4) {
+#pragma unroll
+    for (int i = 0; i < kWideMaxChunks; ++i) {
+      const int c = grp + i * (kWideEpiWarps / 4);
+      if (c >= nu) break;                                    // uniform over the warp
       float v[32];
-      tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), v);
+      tmem_ld32(tlane + (uint32_t)(c * 32), v);
       if (!live) continue;
-      const int nb = n0 + c * 32, j0 = nb >> 2;              // 8 whole hidden units (gate columns interleaved)
-      if (p.bias) {
-#pragma unroll
-        for (int j = 0; j < 32; j += 4) {
-          const float4 b4 = __ldg(reinterpret_cast<const float4*>(p.bias + nb + j));
-          v[j] += b4.x; v[j + 1] += b4.y; v[j + 2] += b4.z; v[j + 3] += b4.w;
-        }
-      }
-      float cp[8];
-      if (wide_ok) {
-        if (arow) {
-#pragma unroll
-          for (int j = 0; j < 32; j += 8) {
-            float a8[8];
-            ld_global_v8(arow + nb + j, a8);
-#pragma unroll
-            for (int u = 0; u < 8; ++u) v[j + u] += a8[u];
-          }
-        }
-        ld_global_v8(cin + j0, cp);
-      } else {
-        if (arow) {
-#pragma unroll
-          for (int j = 0; j < 32; j += 4) {
-            const float4 a4 = __ldg(reinterpret_cast<const float4*>(arow + nb + j));
-            v[j] += a4.x; v[j + 1] += a4.y; v[j + 2] += a4.z; v[j + 3] += a4.w;
-          }
-        }
-        const float4 c0 = *reinterpret_cast<const float4*>(cin + j0), c1 = *reinterpret_cast<const float4*>(cin + j0 + 4);
-        cp[0] = c0.x; cp[1] = c0.y; cp[2] = c0.z; cp[3] = c0.w; cp[4] = c1.x; cp[5] = c1.y; cp[6] = c1.z; cp[7] = c1.w;
-      }
+      const int j0 = (n0 + c * 32) >> 2;
       float hn[8], cn[8];
 #pragma unroll
       for (int u = 0; u < 8; ++u) {
-        const float cc = sigmoid_fast(v[4 * u + 1]) * cp[u] + sigmoid_fast(v[4 * u]) * tanh_fast_g(v[4 * u + 2]);
+        const float cc = sigmoid_fast(v[4 * u + 1]) * cp[i][u] + sigmoid_fast(v[4 * u]) * tanh_fast_g(v[4 * u + 2]);
         cn[u] = cc;
         hn[u] = sigmoid_fast(v[4 * u + 3]) * tanh_fast_g(cc);
       }
@@ -365,7 +393,8 @@ gemm_lstm_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
   uint64_t* full = reinterpret_cast<uint64_t*>(sB + kWideStages * kWideBBytes);
   uint64_t* empty = full + kWideStages;
   uint64_t* acc_full = empty + kWideStages;
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(acc_full + 1);
+  uint64_t* acc_init = acc_full + 1;        // the epilogue warps have written the accumulators' initial values
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(acc_init + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_kb = (p.K + BK - 1) / BK;
@@ -376,6 +405,7 @@ gemm_lstm_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     prefetch_tensormap(&tmB32);
     for (int s = 0; s < kWideStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
     mbar_init(acc_full, 1);
+    mbar_init(acc_init, kWideEpiWarps);
     fence_barrier_init();
     fence_proxy_async_smem();
   }
@@ -422,8 +452,8 @@ gemm_lstm_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     if (lane == 0) {
       const int n1 = w <= 256 ? w : ((w >> 1) + 15) & ~15, n2 = w - n1;    // wider than one MMA: two of about equal width
       const uint32_t idesc1 = make_idesc_bf16(BM, n1), idesc2 = make_idesc_bf16(BM, n2);
-      bool ok = true;
-      for (int kb = 0; kb < num_kb; ++kb) {
+      bool ok = mbar_wait(acc_init, 0, p.err);             // the accumulators hold bias + addend: accumulate onto them
+      for (int kb = 0; kb < num_kb && ok; ++kb) {
         const int s = kb % kWideStages;
         const uint32_t ph = (kb / kWideStages) & 1;
         ok = mbar_wait(&full[s], ph, p.err);
@@ -433,16 +463,16 @@ gemm_lstm_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
 #pragma unroll
         for (int k = 0; k < BK / 16; ++k) {
           const uint64_t da = make_desc_k_sw128(a_addr + k * 32);
-          umma_bf16(tmem_base, da, make_desc_k_sw128(b_addr + k * 32), idesc1, (kb | k) != 0);
+          umma_bf16(tmem_base, da, make_desc_k_sw128(b_addr + k * 32), idesc1, 1u);
           if (n2 > 0)
-            umma_bf16(tmem_base + (uint32_t)n1, da, make_desc_k_sw128(b_addr + n1 * (BK * 2) + k * 32), idesc2, (kb | k) != 0);
+            umma_bf16(tmem_base + (uint32_t)n1, da, make_desc_k_sw128(b_addr + n1 * (BK * 2) + k * 32), idesc2, 1u);
         }
         umma_commit(&empty[s]);
       }
       if (ok) umma_commit(acc_full);
     }
   } else {
-    lstm_tile_epilogue(p, tmem_base, acc_full, M, m0, n0, nu, warp, lane);
+    lstm_tile_epilogue(p, tmem_base, acc_full, acc_init, M, m0, n0, nu, warp, lane);
   }
   tc_fence_before();
   __syncthreads();

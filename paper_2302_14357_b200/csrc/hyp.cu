@@ -9,6 +9,7 @@
 #include <cuda_bf16.h>
 
 #include "tw_internal.cuh"
+#include "sm100.cuh"
 
 namespace tw {
 
@@ -164,7 +165,8 @@ __global__ void __launch_bounds__(2 * kStepThreads) hyp_step_kernel(HypState hs)
       const double base = hs.A_ls[b * kMaxBeam + h];
       // a lower bound of the N-th best value: the N-th largest of the 32 lane maxima (distinct elements)
       float lmax = 0.f;
-      for (int k = lane * 4; k < V; k += 128) {
+#pragma unroll 8
+      for (int k = lane * 4; k < V; k += 128) {             // eight independent loads in flight per lane
         const float4 v = __ldg(reinterpret_cast<const float4*>(src + k));
         lmax = fmaxf(fmaxf(lmax, fmaxf(v.x, v.y)), fmaxf(v.z, v.w));
       }
@@ -176,14 +178,27 @@ __global__ void __launch_bounds__(2 * kStepThreads) hyp_step_kernel(HypState hs)
       for (int j = 0; j < 32; ++j) { const float o = s_lm[h][j]; lrank += (o > lmax || (o == lmax && j < lane)) ? 1 : 0; }
       const unsigned who = __ballot_sync(0xffffffffu, lrank == N - 1);        // exactly one lane: the ranks are 0..31
       const float bound = __shfl_sync(0xffffffffu, lmax, __ffs(who) - 1);
-      for (int k = lane * 4; k < V; k += 128) {
-        const float4 v4 = __ldg(reinterpret_cast<const float4*>(src + k));
-        const float vv[4] = {v4.x, v4.y, v4.z, v4.w};
+      // second sweep (the row is in L2): eight loads at a time, and only a group of four that holds a survivor
+      // enters the branch with the shared-memory counter
+      for (int k0 = lane * 4; k0 < V; k0 += 8 * 128) {
+        float4 v8[8];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          if (vv[c] >= bound && vv[c] > 0.f) {
-            const int i = atomicAdd(&s_cnt[h], 1);
-            if (i < kSelCap) { s_sv[h][i] = vv[c]; s_sk[h][i] = k + c; }
+        for (int u = 0; u < 8; ++u) {
+          const int k = k0 + u * 128;
+          v8[u] = k < V ? __ldg(reinterpret_cast<const float4*>(src + k)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const float g = fmaxf(fmaxf(v8[u].x, v8[u].y), fmaxf(v8[u].z, v8[u].w));
+          if (g >= bound && g > 0.f) {
+            const float vv[4] = {v8[u].x, v8[u].y, v8[u].z, v8[u].w};
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              if (vv[c] >= bound && vv[c] > 0.f) {
+                const int i = atomicAdd(&s_cnt[h], 1);
+                if (i < kSelCap) { s_sv[h][i] = vv[c]; s_sk[h][i] = k0 + u * 128 + c; }
+              }
+            }
           }
         }
       }
@@ -423,6 +438,11 @@ __global__ void __launch_bounds__(2 * kStepThreads) hyp_step_kernel(HypState hs)
       hs.A_ls[b * kMaxBeam + i] = s_keep_ls[i];
     }
     if (hs.inline_gather && lane == 0) {           // the predictor's work-list entry of this hypothesis
+      if (hs.pf_table != nullptr) sm100::prefetch_l2_bulk(hs.pf_table + (long long)k * hs.pf_row_bytes, (uint32_t)hs.pf_row_bytes);
+      if ((hs.Hd & 3) == 0) {
+        const float* pc = hs.slot_hc + gp * ((long long)hs.L * 2 * hs.Hd) + hs.Hd;      // the parent's c, layer by layer
+        for (int l = 0; l < hs.L; ++l) sm100::prefetch_l2_bulk(pc + (long long)l * 2 * hs.Hd, (uint32_t)hs.Hd * 4u);
+      }
       const int wrow = s_wbase + i;
       if (wrow < hs.B * hs.N) { hs.pw_new[wrow] = (int)gn; hs.pw_par[wrow] = (int)gp; hs.pw_tok[wrow] = k; }
       else hs.status[b] = TW_ERR_LIMIT;            // cannot happen: the list holds at most N entries per utterance
@@ -630,6 +650,16 @@ __global__ void lstm_pointwise_kernel(const float* gates, const int* pw_new, con
 }
 
 }  // namespace
+
+// The kernels of a decode step alternate with GEMM kernels that take nearly all of an SM's shared memory.  An SM whose
+// shared-memory / L1 split differs from what the next kernel asks for is drained and reconfigured before that kernel's
+// CTAs start; these kernels hardly use L1, so they ask for the same (largest) shared-memory carve-out.
+int hyp_setup() {
+  const int mx = (int)cudaSharedmemCarveoutMaxShared;
+  cudaError_t e1 = cudaFuncSetAttribute(hyp_step_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, mx);
+  cudaError_t e2 = cudaFuncSetAttribute(compact_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, mx);
+  return (e1 == cudaSuccess && e2 == cudaSuccess) ? TW_OK : TW_ERR_CUDA;
+}
 
 void launch_hyp_init(const HypState& hs, const int* lengths, int B, int T, cudaStream_t st) {
   if (B > 0) hyp_init_kernel<<<B, kThreads, 0, st>>>(hs, lengths, T);

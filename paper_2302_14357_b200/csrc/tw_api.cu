@@ -272,6 +272,10 @@ int build_bf16(tw_handle* h) {
     // hyp_step_kernel builds the predictor's work list and operand rows itself (HypState::inline_gather)
     if (h->hs_fused.defer_rows && h->pred_kind != TW_PRED_STATELESS) {
       h->hs_fused.inline_gather = 1;
+      if ((((size_t)4 * h->Hd * sizeof(float)) & 15) == 0) {
+        h->hs_fused.pf_table = reinterpret_cast<const char*>(h->bf.EmbProj);
+        h->hs_fused.pf_row_bytes = 4 * h->Hd * (int)sizeof(float);
+      }
       for (int l = 0; l < h->L; ++l) {
         h->hs_fused.xg_dst[l] = h->bf.X[l].ptr; h->hs_fused.xg_ld[l] = (int)h->bf.X[l].K; h->hs_fused.xg_off[l] = (l == 0) ? 0 : h->Hd;
       }
@@ -371,6 +375,7 @@ int init_impl(tw_handle* h, const tw_model* m, const tw_config* c) {
     TW_TRY(copy_weight(h, &h->W_hh[l], m->host_lstm_W_hh[l], (size_t)4 * h->Hd * h->Hd));
     TW_TRY(copy_weight(h, &h->b_l[l], m->host_lstm_b[l], (size_t)4 * h->Hd));
   }
+  TW_TRY(hyp_setup());
   TW_TRY(build_workspace(h));
   if (h->mode == TW_MODE_BF16) TW_TRY(build_bf16(h));
 
@@ -457,7 +462,7 @@ int enqueue_joiner_fused(tw_handle* h, const JoinerRows& rows, const float* ld_o
   {
     PdlScope first(plain_first ? false : g_pdl_on);
     if (utt_B > 0) launch_joiner_A_tiled_utt(rows, h->hs.row_off, h->hs.nA, utt_B, h->bf.A_tiled.ptr, st);
-    else launch_joiner_A_tiled(rows, h->bf.A_tiled.ptr, st);
+    else launch_joiner_A_tiled(rows, h->bf.A_tiled.ptr, st, h->bf.W_out_pad.ptr, (long long)h->bf.W_out_pad.rows * h->bf.W_out_pad.K * 2);
   }
   if (mark_fn) mark_fn(h, 3, st);       // operand preparation is booked with the elementwise stages
   if (ldnb == nullptr) ldnb = h->bf.ldnb_pad;   // a caller's buffer has V columns: only with an unpadded vocabulary

@@ -195,8 +195,13 @@ struct HypState {
   // from run to run; no result depends on it (every entry is computed on its own).
   int inline_gather;
   void* xg_dst[kMaxLayers]; int xg_ld[kMaxLayers]; int xg_off[kMaxLayers];
+  // With inline_gather: the first gate GEMM adds a row of this table per new hypothesis ([V] rows of pf_row_bytes, a
+  // table far larger than L2) and every layer reads the parent's cell state; hyp_step_kernel, which is the first to
+  // know tokens and parents, asks for both in L2 so that the GEMM's epilogue threads do not each wait on DRAM.
+  const char* pf_table; int pf_row_bytes;
 };
 
+int hyp_setup();   // once per process: kernel attributes
 void launch_hyp_init(const HypState& hs, const int* lengths, int B, int T, cudaStream_t st);
 void launch_hyp_step(const HypState& hs, int B, cudaStream_t st);
 void launch_compact(const HypState& hs, int B, int T, cudaStream_t st);
