@@ -462,7 +462,11 @@ int enqueue_joiner_fused(tw_handle* h, const JoinerRows& rows, const float* ld_o
   {
     PdlScope first(plain_first ? false : g_pdl_on);
     if (utt_B > 0) launch_joiner_A_tiled_utt(rows, h->hs.row_off, h->hs.nA, utt_B, h->bf.A_tiled.ptr, st);
-    else launch_joiner_A_tiled(rows, h->bf.A_tiled.ptr, st, h->bf.W_out_pad.ptr, (long long)h->bf.W_out_pad.rows * h->bf.W_out_pad.K * 2);
+    else {
+      // a small model's weights stay in L2 between two steps by themselves; a large one's W_out is asked for again
+      const long long wbytes = (long long)h->bf.W_out_pad.rows * h->bf.W_out_pad.K * 2;
+      launch_joiner_A_tiled(rows, h->bf.A_tiled.ptr, st, wbytes >= (4ll << 20) ? h->bf.W_out_pad.ptr : nullptr, wbytes);
+    }
   }
   if (mark_fn) mark_fn(h, 3, st);       // operand preparation is booked with the elementwise stages
   if (ldnb == nullptr) ldnb = h->bf.ldnb_pad;   // a caller's buffer has V columns: only with an unpadded vocabulary
