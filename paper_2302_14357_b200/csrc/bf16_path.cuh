@@ -99,6 +99,8 @@ struct FusedJoinerParams {
   const int* row_slen;               // [R] (nullptr: S)
   float* ldphi; float* la; float* lse;   // [R], [R][S], [R][S]
   float* ldnb;                       // [R][V] delta_nb as a probability ratio, NOT its log (0 at the blank column)
+  float* dmax;                       // optional [R][V / 32]: the largest delta_nb of every 32-column chunk of every row
+                                     // (written by the instances that sum over frames with shuffles: fused_joiner_writes_maxima)
   int* err;
   int hat;                           // factorised output (JoinerRows::hat); log2_tau = log2 of the blank threshold
   float log2_tau;
@@ -106,7 +108,8 @@ struct FusedJoinerParams {
   int* clear_word;                   // optional: one device word the kernel sets to 0 once its predecessors have finished
 };
 bool fused_joiner_eligible(int S, int V, int J);
-bool fused_joiner_specialised(int S);   // a kernel instance with this segment size compiled in exists
+bool fused_joiner_specialised(int S);
+bool fused_joiner_writes_maxima(int S);   // the instance for this segment size fills FusedJoinerParams::dmax   // a kernel instance with this segment size compiled in exists
 long long fused_joiner_A_rows(int R_max, int S);      // rows of the tile-layout A operand
 int fused_joiner_setup(int CL, int S, int* max_clusters);
 // max_k (sum_j |W_out[k, j]| + |b_out[k]|): bound of |z| since |tanh| <= 1; written to *out (device)

@@ -164,11 +164,23 @@ __global__ void __launch_bounds__(2 * kStepThreads) hyp_step_kernel(HypState hs)
       const float* src = hs.dnb_sel + (long long)(r0 + h) * V;
       const double base = hs.A_ls[b * kMaxBeam + h];
       // a lower bound of the N-th best value: the N-th largest of the 32 lane maxima (distinct elements)
+      const int nchunk = V >> 5;
+      const float* cmax = (hs.dnb_max != nullptr && (V & 31) == 0 && nchunk <= 128) ? hs.dnb_max + (long long)(r0 + h) * nchunk : nullptr;
       float lmax = 0.f;
+      float m4[4] = {0.f, 0.f, 0.f, 0.f};        // with chunk maxima: those of chunks lane, lane + 32, lane + 64, lane + 96
+      if (cmax != nullptr) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int c = lane + 32 * u;
+          if (c < nchunk) m4[u] = __ldg(cmax + c);
+          lmax = fmaxf(lmax, m4[u]);
+        }
+      } else {
 #pragma unroll 8
-      for (int k = lane * 4; k < V; k += 128) {             // eight independent loads in flight per lane
-        const float4 v = __ldg(reinterpret_cast<const float4*>(src + k));
-        lmax = fmaxf(fmaxf(lmax, fmaxf(v.x, v.y)), fmaxf(v.z, v.w));
+        for (int k = lane * 4; k < V; k += 128) {             // eight independent loads in flight per lane
+          const float4 v = __ldg(reinterpret_cast<const float4*>(src + k));
+          lmax = fmaxf(fmaxf(lmax, fmaxf(v.x, v.y)), fmaxf(v.z, v.w));
+        }
       }
       s_lm[h][lane] = lmax;
       if (lane == 0) s_cnt[h] = 0;
@@ -178,27 +190,60 @@ __global__ void __launch_bounds__(2 * kStepThreads) hyp_step_kernel(HypState hs)
       for (int j = 0; j < 32; ++j) { const float o = s_lm[h][j]; lrank += (o > lmax || (o == lmax && j < lane)) ? 1 : 0; }
       const unsigned who = __ballot_sync(0xffffffffu, lrank == N - 1);        // exactly one lane: the ranks are 0..31
       const float bound = __shfl_sync(0xffffffffu, lmax, __ffs(who) - 1);
-      // second sweep (the row is in L2): eight loads at a time, and only a group of four that holds a survivor
-      // enters the branch with the shared-memory counter
-      for (int k0 = lane * 4; k0 < V; k0 += 8 * 128) {
-        float4 v8[8];
+      auto push4 = [&](const float4& v4, int k) {
+        const float vv[4] = {v4.x, v4.y, v4.z, v4.w};
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          const int k = k0 + u * 128;
-          v8[u] = k < V ? __ldg(reinterpret_cast<const float4*>(src + k)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int c = 0; c < 4; ++c) {
+          if (vv[c] >= bound && vv[c] > 0.f) {
+            const int i = atomicAdd(&s_cnt[h], 1);
+            if (i < kSelCap) { s_sv[h][i] = vv[c]; s_sk[h][i] = k + c; }
+          }
         }
+      };
+      if (cmax != nullptr) {
+        // Only the chunks whose maximum reaches the bound can hold a survivor: a few 128-byte pieces of the row.  The
+        // warp takes them together, a lane per element and up to eight chunks per round, so that their loads (mostly
+        // from DRAM: a step moves more than L2 holds) are in flight at the same time.
+        unsigned qm[4];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          const float g = fmaxf(fmaxf(v8[u].x, v8[u].y), fmaxf(v8[u].z, v8[u].w));
-          if (g >= bound && g > 0.f) {
-            const float vv[4] = {v8[u].x, v8[u].y, v8[u].z, v8[u].w};
+        for (int u = 0; u < 4; ++u) qm[u] = __ballot_sync(0xffffffffu, m4[u] >= bound && m4[u] > 0.f);
+        int u = 0;
+        unsigned m = qm[0];
+        for (;;) {
+          int ids[8];
+          int n = 0;
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-              if (vv[c] >= bound && vv[c] > 0.f) {
-                const int i = atomicAdd(&s_cnt[h], 1);
-                if (i < kSelCap) { s_sv[h][i] = vv[c]; s_sk[h][i] = k0 + u * 128 + c; }
-              }
+          for (int x = 0; x < 8; ++x) {
+            while (m == 0u && u < 3) { ++u; m = (u == 1) ? qm[1] : (u == 2 ? qm[2] : qm[3]); }
+            ids[x] = -1;
+            if (m != 0u) { ids[x] = (__ffs(m) - 1) + 32 * u; m &= m - 1; ++n; }
+          }
+          if (n == 0) break;
+          float v[8];
+#pragma unroll
+          for (int x = 0; x < 8; ++x) v[x] = ids[x] >= 0 ? __ldg(src + ids[x] * 32 + lane) : 0.f;
+#pragma unroll
+          for (int x = 0; x < 8; ++x) {
+            if (v[x] >= bound && v[x] > 0.f) {
+              const int i = atomicAdd(&s_cnt[h], 1);
+              if (i < kSelCap) { s_sv[h][i] = v[x]; s_sk[h][i] = ids[x] * 32 + lane; }
             }
+          }
+        }
+      } else {
+        // second sweep (the row is in L2): eight loads at a time, and only a group of four that holds a survivor
+        // enters the branch with the shared-memory counter
+        for (int k0 = lane * 4; k0 < V; k0 += 8 * 128) {
+          float4 v8[8];
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            const int k = k0 + u * 128;
+            v8[u] = k < V ? __ldg(reinterpret_cast<const float4*>(src + k)) : make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            const float g = fmaxf(fmaxf(v8[u].x, v8[u].y), fmaxf(v8[u].z, v8[u].w));
+            if (g >= bound && g > 0.f) push4(v8[u], k0 + u * 128);
           }
         }
       }

@@ -249,6 +249,7 @@ int build_bf16(tw_handle* h) {
       h->bf.zbound = bound;
       TW_TRY(make_bf16_mat(h, &h->bf.A_tiled, nullptr, fused_joiner_A_rows(h->R_max, h->S), h->J, true, false));
       TW_TRY(dev_alloc(h, &h->bf.lse, (size_t)h->R_max * h->S));
+      TW_TRY(dev_alloc(h, &h->bf.dmax, (size_t)h->R_max * (h->bf.Vp / 32)));
       TW_TRY(scan_select_setup());
       h->bf.fused_ok = true;
       // default: on for the segment sizes with a specialised kernel instance; the generic instance is
@@ -259,6 +260,7 @@ int build_bf16(tw_handle* h) {
   h->hs.defer_rows = 0;
   h->hs.inline_gather = 0;
   h->hs.dnb_sel = nullptr;
+  h->hs.dnb_max = nullptr;
   h->hs_fused = h->hs;
   h->hs_fused.logp = nullptr; h->hs_fused.lse = nullptr; h->hs_fused.ldphi_d = nullptr; h->hs_fused.la_d = nullptr;
   if (h->mode == TW_MODE_BF16 && h->bf.fused_ok) {
@@ -268,6 +270,7 @@ int build_bf16(tw_handle* h) {
     if (!h->aux_ok) cudaGetLastError();
     h->hs_fused.defer_rows = h->aux_ok ? 1 : 0;
     h->hs_fused.dnb_sel = h->bf.ldnb_pad;        // the step's hyp_step_kernel picks the rows' best tokens itself
+    h->hs_fused.dnb_max = fused_joiner_writes_maxima(h->S) ? h->bf.dmax : nullptr;
     h->hs_fused.V = h->bf.Vp;                    // row pitch of delta_nb there (padding columns hold 0)
     // hyp_step_kernel builds the predictor's work list and operand rows itself (HypState::inline_gather)
     if (h->hs_fused.defer_rows && h->pred_kind != TW_PRED_STATELESS) {
@@ -474,6 +477,7 @@ int enqueue_joiner_fused(tw_handle* h, const JoinerRows& rows, const float* ld_o
   fp.R_dev = rows.R_dev; fp.R_max = rows.R_max; fp.S = rows.S; fp.V = h->bf.Vp; fp.K = rows.J; fp.blank = h->blank;
   fp.CL = h->bf.CL; fp.no_max = h->bf.no_max ? 1 : 0; fp.zbound = h->bf.zbound; fp.bias = h->bf.bias_pad; fp.ld_old = ld_old; fp.row_slen = rows.row_slen;
   fp.ldphi = ldphi; fp.la = la; fp.lse = h->bf.lse; fp.ldnb = ldnb; fp.err = h->bf.err; fp.clear_word = clear_word;
+  fp.dmax = (ldnb == h->bf.ldnb_pad && fused_joiner_writes_maxima(rows.S)) ? h->bf.dmax : nullptr;   // the chunk maxima belong to the handle's own delta_nb buffer
   fp.hat = rows.hat; fp.log2_tau = rows.log_tau * 1.4426950408889634f; fp.skipped = rows.skipped;
   TW_TRY(launch_fused_joiner(h->bf.A_tiled.as_A, h->bf.W_out_pad.as_B256, fp, h->bf.max_clusters, st));
   if (mark_fn) mark_fn(h, 2, st);       // the fused kernel alone

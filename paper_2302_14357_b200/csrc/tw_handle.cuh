@@ -54,6 +54,7 @@ struct tw_handle {
     tw::Bf16Mat W_out_pad;
     float* bias_pad = nullptr;
     float* ldnb_pad = nullptr;                            // [R_max, Vp]
+    float* dmax = nullptr;                                // [R_max, Vp / 32] chunk maxima of delta_nb (fused decode path)
     tw::Bf16Mat A_tiled;                                  // A operand in the fused kernel's tile layout
     float* lse = nullptr;                                 // [R_max, S]
   } bf;

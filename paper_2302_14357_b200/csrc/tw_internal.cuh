@@ -163,6 +163,9 @@ struct HypState {
   // dnb_sel != nullptr: delta_nb [R][V] as plain probability ratios (0: no candidate); hyp_step_kernel then picks
   // every row's N best tokens itself instead of reading cand_v / cand_k / cand_n
   const float* dnb_sel;
+  // with dnb_sel: optional [R][V / 32] largest value of every 32-column chunk of a row, written by the kernel that wrote
+  // delta_nb; the selection then reads these first and only the few chunks that can hold one of the N best after them
+  const float* dnb_max;
   // list B of Algorithm 1 (hypotheses finished for this segment): [B][capB]
   int* B_slot; double* B_ls; unsigned long long* B_hash; int* B_len;
   int* B_top;    // [B][kMaxBeam] indices into list B of its best entries, best first
