@@ -137,10 +137,21 @@ __global__ void __launch_bounds__(2 * kStepThreads) hyp_step_kernel(HypState hs)
     if (hs.mono) ld_Adone = hs.A_done[b * kMaxBeam + tid];
     ld_carry = hs.carry[b * kMaxBeam + tid];
   }
-  if (H == 0) return;                       // idle (finished) utterance
-  const int N = hs.N, S = hs.S, V = hs.V;
   const long long bB = (long long)b * hs.capB;
   const long long bS = (long long)b * hs.capSlot;
+  // the search of list B (warp h looks for hypothesis h's tokens): its own slot and the first 32 entries of the list are
+  // asked for now as well; the slot's hash and length follow as soon as the slot is there, still before the barriers
+  int my_slot = 0, pre_len = -1, pre_slot = 0;
+  unsigned long long pre_hash = 0;
+  if (warp < kMaxBeam) {
+    my_slot = hs.A_slot[b * kMaxBeam + warp];
+    if (lane < hs.capB) { pre_hash = hs.B_hash[bB + lane]; pre_len = hs.B_len[bB + lane]; pre_slot = hs.B_slot[bB + lane]; }
+  }
+  if (H == 0) return;                       // idle (finished) utterance
+  const int N = hs.N, S = hs.S, V = hs.V;
+  unsigned long long my_hash = 0;
+  int my_len = 0;
+  if (warp < H) { my_hash = hs.slot_hash[bS + my_slot]; my_len = hs.slot_len[bS + my_slot]; }
 
   if (tid < kMaxBeam) { s_Als[tid] = ld_Als; s_Aslot[tid] = ld_Aslot; s_Adone[tid] = ld_Adone; s_carry[tid] = ld_carry; }
   if (tid == 0) { hs.calls[b] += 1; hs.joins[b] += slen; }
@@ -305,19 +316,20 @@ __global__ void __launch_bounds__(2 * kStepThreads) hyp_step_kernel(HypState hs)
   // ---- AddAndMerge, search: warp h looks for the tokens of A_h among the entries already in B.
   // (Entries of A are distinct sequences, so two of them never merge with each other.)
   if (warp < H) {
-    const int slot = s_Aslot[warp];
-    const unsigned long long hh = hs.slot_hash[bS + slot];
-    const int ln = hs.slot_len[bS + slot];
+    const int slot = my_slot;
+    const unsigned long long hh = my_hash;
+    const int ln = my_len;
     const int* ta = hs.slot_tok + (bS + slot) * hs.U_cap;
     int found = -1;
     for (int base = 0; base < nB0 && found < 0; base += 32) {
       const int e = base + lane;
-      const bool match = e < nB0 && hs.B_hash[bB + e] == hh && hs.B_len[bB + e] == ln;
+      const bool match = e < nB0 && (base == 0 ? (pre_hash == hh && pre_len == ln)
+                                               : (hs.B_hash[bB + e] == hh && hs.B_len[bB + e] == ln));
       unsigned mask = __ballot_sync(0xffffffffu, match);
       while (mask != 0 && found < 0) {
         const int c = base + __ffs(mask) - 1;
         mask &= mask - 1;
-        const int oslot = hs.B_slot[bB + c];
+        const int oslot = base == 0 ? __shfl_sync(0xffffffffu, pre_slot, c) : hs.B_slot[bB + c];
         int diff = 0;                       // a 64-bit hash match is not proof: compare the tokens
         if (oslot != slot) {
           const int* tb = hs.slot_tok + (bS + oslot) * hs.U_cap;
@@ -695,16 +707,6 @@ __global__ void lstm_pointwise_kernel(const float* gates, const int* pw_new, con
 }
 
 }  // namespace
-
-// The kernels of a decode step alternate with GEMM kernels that take nearly all of an SM's shared memory.  An SM whose
-// shared-memory / L1 split differs from what the next kernel asks for is drained and reconfigured before that kernel's
-// CTAs start; these kernels hardly use L1, so they ask for the same (largest) shared-memory carve-out.
-int hyp_setup() {
-  const int mx = (int)cudaSharedmemCarveoutMaxShared;
-  cudaError_t e1 = cudaFuncSetAttribute(hyp_step_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, mx);
-  cudaError_t e2 = cudaFuncSetAttribute(compact_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, mx);
-  return (e1 == cudaSuccess && e2 == cudaSuccess) ? TW_OK : TW_ERR_CUDA;
-}
 
 void launch_hyp_init(const HypState& hs, const int* lengths, int B, int T, cudaStream_t st) {
   if (B > 0) hyp_init_kernel<<<B, kThreads, 0, st>>>(hs, lengths, T);

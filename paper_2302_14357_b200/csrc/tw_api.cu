@@ -378,7 +378,6 @@ int init_impl(tw_handle* h, const tw_model* m, const tw_config* c) {
     TW_TRY(copy_weight(h, &h->W_hh[l], m->host_lstm_W_hh[l], (size_t)4 * h->Hd * h->Hd));
     TW_TRY(copy_weight(h, &h->b_l[l], m->host_lstm_b[l], (size_t)4 * h->Hd));
   }
-  TW_TRY(hyp_setup());
   TW_TRY(build_workspace(h));
   if (h->mode == TW_MODE_BF16) TW_TRY(build_bf16(h));
 

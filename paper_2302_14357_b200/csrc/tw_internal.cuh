@@ -204,7 +204,6 @@ struct HypState {
   const char* pf_table; int pf_row_bytes;
 };
 
-int hyp_setup();   // once per process: kernel attributes
 void launch_hyp_init(const HypState& hs, const int* lengths, int B, int T, cudaStream_t st);
 void launch_hyp_step(const HypState& hs, int B, cudaStream_t st);
 void launch_compact(const HypState& hs, int B, int T, cudaStream_t st);
