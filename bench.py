@@ -51,12 +51,14 @@ def parse_args():
 
 
 # DRAM traffic of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum per launch) from ncu captures
-# of this same kernel: "cold" is the first launches of a process, "warm" a launch inside a running decode.  Each
+# of this same kernel: "cold" with the caches flushed before the launch (ncu's default), "warm" with the caches as
+# the running decode leaves them (--cache-control none); the commands are in profiles/.  Each
 # entry carries the digest of the kernel's sources at the time of the capture; once the sources differ the
 # counters no longer describe the kernel that runs and the bench reports null.
 KERNEL_SOURCES = ("fused_joiner.cu", "fused_joiner_kernel.inc", "fused_joiner_host.inc", "sm100.cuh")
 NCU_DRAM_BYTES_PER_LAUNCH = {
     # (workload, S): (source digest, cold bytes, warm bytes)
+    ("c3", 3): ("ad65add11c7b", 16881000, 14732000),      # cold: W_out + the A operand; warm: 2.0 MB read, 12.7 MB of delta_nb leaving L2
 }
 
 
