@@ -111,6 +111,13 @@ def test_fused_joiner_c3_step_shape_every_element():
     _run(cfg, S=3, N=10, R=1275, G=128, seed=31)
 
 
+def test_fused_joiner_two_frame_segments_every_element():
+    """S = 2 on the c3 model: 64 hypotheses per tile, 24 tiles on the 7 resident clusters (the two lanes of a
+    hypothesis share out the columns of delta_nb between them)."""
+    cfg = tw_synth.get_config("c3")
+    _run(cfg, S=2, N=10, R=1500, G=150, seed=36)
+
+
 def test_fused_joiner_c4_step_shape_every_element():
     """S = 10 (the staged sums over a hypothesis's frames), V = 4096, J = 1024, 2590 rows: 216 tiles of 12
     hypotheses, 31 rounds on 7 clusters, the last one ragged."""
