@@ -31,6 +31,8 @@ struct GemmBf16Params {
   const int* add_idx = nullptr;
   long long ld_add = 0;
   int epi = 0;        // 0: store C (+ bias, + addend); 1: LSTM cell (C is not written)
+  int m_early = 0;    // 1: *M_dev was written before the kernel launched ahead of this one began (not by that kernel):
+                      // it is read during the set-up, ahead of the wait for that kernel
   LstmEpi lstm = {};
 };
 

@@ -50,6 +50,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_kb = (p.K + BK - 1) / BK;
+  const int M_pre = (p.m_early && p.M_dev) ? __ldcg(p.M_dev) : 0;   // under the set-up's latency (see m_early)
 
   if (threadIdx.x == 0) {
     prefetch_tensormap(&tmA);
@@ -67,7 +68,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   // the set-up above touched only this CTA: it may overlap the tail of the kernel that produces A and M
   pdl_wait();
   pdl_trigger();
-  const int M = p.M_dev ? *p.M_dev : p.M;
+  const int M = p.M_dev ? (p.m_early ? M_pre : *p.M_dev) : p.M;
   const int m_tiles = (M + BM - 1) / BM, n_tiles = (p.N + BN - 1) / BN;
   const int num_tiles = m_tiles * n_tiles;     // a CTA past the last tile runs no loop iteration below
 
@@ -398,6 +399,7 @@ gemm_lstm_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_kb = (p.K + BK - 1) / BK;
+  const int M_pre = (p.m_early && p.M_dev) ? __ldcg(p.M_dev) : 0;   // under the set-up's latency (see m_early)
 
   if (threadIdx.x == 0) {
     prefetch_tensormap(&tmA);
@@ -419,7 +421,7 @@ gemm_lstm_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
   pdl_trigger();
   // The split follows the row count of THIS launch: fewer row tiles than the grid was sized for give
   // every row tile more CTAs, i.e. narrower and faster tiles (never wider than the host's bound).
-  const int M = p.M_dev ? *p.M_dev : p.M;
+  const int M = p.M_dev ? (p.m_early ? M_pre : *p.M_dev) : p.M;
   const int m_tiles = M > 0 ? (M + BM - 1) / BM : 1;
   const int units = p.N >> 5;
   int n_split = (int)gridDim.x / m_tiles;

@@ -121,11 +121,12 @@ __global__ void __launch_bounds__(2 * kStepThreads) hyp_step_kernel(HypState hs)
   __shared__ int s_keep_h[kMaxBeam], s_keep_k[kMaxBeam], s_keep_slot[kMaxBeam];
   __shared__ double s_keep_ls[kMaxBeam];
 
-  pdl_wait();
-  pdl_trigger();
   const int b = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  // every first-round load is issued before the early exit below, so that none of them waits for H
+  // The lists and counters read below were written by the previous pass's kernels, all of which had finished before
+  // the joiner kernel that runs ahead of this one began (and that kernel writes none of them): they are fetched
+  // before the wait for it, under its tail.  Every first-round load is issued before the early exit, so that none
+  // of them waits for H.
   const int H = hs.nA[b];
   const int r0 = hs.row_off[b];
   const int slen = hs.slen[b];
@@ -147,11 +148,13 @@ __global__ void __launch_bounds__(2 * kStepThreads) hyp_step_kernel(HypState hs)
     my_slot = hs.A_slot[b * kMaxBeam + warp];
     if (lane < hs.capB) { pre_hash = hs.B_hash[bB + lane]; pre_len = hs.B_len[bB + lane]; pre_slot = hs.B_slot[bB + lane]; }
   }
-  if (H == 0) return;                       // idle (finished) utterance
-  const int N = hs.N, S = hs.S, V = hs.V;
   unsigned long long my_hash = 0;
   int my_len = 0;
   if (warp < H) { my_hash = hs.slot_hash[bS + my_slot]; my_len = hs.slot_len[bS + my_slot]; }
+  pdl_wait();                               // from here on: what the joiner kernel wrote (delta_phi, delta_nb, occupancies)
+  pdl_trigger();
+  if (H == 0) return;                       // idle (finished) utterance
+  const int N = hs.N, S = hs.S, V = hs.V;
 
   if (tid < kMaxBeam) { s_Als[tid] = ld_Als; s_Aslot[tid] = ld_Aslot; s_Adone[tid] = ld_Adone; s_carry[tid] = ld_carry; }
   if (tid == 0) { hs.calls[b] += 1; hs.joins[b] += slen; }

@@ -74,9 +74,9 @@ int make_bf16_mat(tw_handle* h, Bf16Mat* m, const float* src, long long rows, lo
 
 void gemm_bf16(tw_handle* h, const Bf16Mat& A, const Bf16Mat& B, const int* M_dev, int M, float* C, const int* oidx,
                long long ldC, const float* bias, cudaStream_t st, const float* addend = nullptr,
-               const int* add_idx = nullptr, long long ld_add = 0) {
+               const int* add_idx = nullptr, long long ld_add = 0, int m_early = 0) {
   GemmBf16Params p{M_dev, M, (int)B.rows, (int)A.K, C, oidx, ldC, bias, h->bf.err};
-  p.addend = addend; p.add_idx = add_idx; p.ld_add = ld_add;
+  p.addend = addend; p.add_idx = add_idx; p.ld_add = ld_add; p.m_early = m_early;
   launch_gemm_bf16(A.as_A, B.as_B128, B.as_B256, p, st, &B.as_B64);
 }
 
@@ -109,12 +109,13 @@ void enqueue_predictor(tw_handle* h, const int* tok, const float* hc_in, const i
       if (l == 0) { p.addend = h->bf.EmbProj; p.add_idx = tok; p.ld_add = 4 * Hd; }   // W_ih[0] emb[tok] + b[0]: a table row
       else p.bias = h->bf.bias_perm[l];
       p.epi = 1;
+      p.m_early = l > 0;                      // the row count is older than the layer below, which runs ahead of this one
       p.lstm = LstmEpi{hc_in, idx_in, hc_out, idx_out, L, l, Hd,
                        (l + 1 < L) ? h->bf.X[l + 1].ptr : h->bf.Htop.ptr, (l + 1 < L) ? 2LL * Hd : (long long)Hd};
       if (!launch_gemm_lstm_wide(h->bf.X[l].as_A, h->bf.W_cat[l].as_B64, h->bf.W_cat[l].as_B32, p, st))
         launch_gemm_bf16(h->bf.X[l].as_A, h->bf.W_cat[l].as_B128, h->bf.W_cat[l].as_B256, p, st);
     }
-    gemm_bf16(h, h->bf.Htop, h->bf.W_p, n_dev, n_max, Pp_out, idx_out, h->J, nullptr, st);
+    gemm_bf16(h, h->bf.Htop, h->bf.W_p, n_dev, n_max, Pp_out, idx_out, h->J, nullptr, st, nullptr, nullptr, 0, /*m_early=*/1);
     *launches += L + (gathered ? 1 : 2);
     return;
   }
