@@ -92,7 +92,8 @@ void launch_joiner_A_bf16(const JoinerRows& rows, __nv_bfloat16* A, cudaStream_t
 
 // ---- fused joiner + softmax + Eq. 3-7 + candidate selection (fused_joiner.cu) ------------------
 struct FusedJoinerParams {
-  const int* R_dev; int R_max;       // hypothesis rows (device count optional)
+  const int* R_dev; int R_max;       // hypothesis rows (device count optional; written before the operand kernel ahead of this
+                                     // one was launched, and not by it: the kernel reads it ahead of its wait)
   int S, V, K, blank, CL;            // CL = V / 256 CTAs per cluster; K = J
   int no_max;                        // logits are bounded by zbound (at most 40): softmax sums need no maximum search
   float zbound;                      // max_k (|W_out[k, :]|_1 + |b_out[k]|) >= |z| (tanh joiner); used when no_max
@@ -108,6 +109,7 @@ struct FusedJoinerParams {
   float log2_tau;
   unsigned long long* skipped;       // optional counter of the (row, frame) pairs blank thresholding left out
   int* clear_word;                   // optional: one device word the kernel sets to 0 once its predecessors have finished
+  int early_w;                       // 1: the W_out tiles of the first ring stages are asked for ahead of the wait for the operand kernel
 };
 bool fused_joiner_eligible(int S, int V, int J);
 bool fused_joiner_specialised(int S);

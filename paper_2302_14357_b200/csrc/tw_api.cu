@@ -478,6 +478,7 @@ int enqueue_joiner_fused(tw_handle* h, const JoinerRows& rows, const float* ld_o
   fp.CL = h->bf.CL; fp.no_max = h->bf.no_max ? 1 : 0; fp.zbound = h->bf.zbound; fp.bias = h->bf.bias_pad; fp.ld_old = ld_old; fp.row_slen = rows.row_slen;
   fp.ldphi = ldphi; fp.la = la; fp.lse = h->bf.lse; fp.ldnb = ldnb; fp.err = h->bf.err; fp.clear_word = clear_word;
   fp.dmax = (ldnb == h->bf.ldnb_pad && fused_joiner_writes_maxima(rows.S)) ? h->bf.dmax : nullptr;   // the chunk maxima belong to the handle's own delta_nb buffer
+  fp.early_w = utt_B > 0 ? 0 : 1;       // (measured: beside the per-utterance operand kernel the early loads cost 6 % at c2, S = 10)
   fp.hat = rows.hat; fp.log2_tau = rows.log_tau * 1.4426950408889634f; fp.skipped = rows.skipped;
   TW_TRY(launch_fused_joiner(h->bf.A_tiled.as_A, h->bf.W_out_pad.as_B256, fp, h->bf.max_clusters, st));
   if (mark_fn) mark_fn(h, 2, st);       // the fused kernel alone
