@@ -411,7 +411,10 @@ def run_ours(args, cfg, S):
                      "unit": "TFLOP/s", "frac": achieved / peak if peak else None,
                      "frac_sustained": achieved / peaks["tflops_sustained"], "frac_burst": achieved / peaks["tflops_burst"],
                      "peak_burst": peaks["tflops_burst"],
-                     "traffic": traffic, "traffic_kernel_digest": traffic_rev,
+                     # bytes per launch: the ncu capture with the caches flushed before the launch (the profiling
+                     # recipe's); traffic_warm: with the caches as the running decode leaves them
+                     "traffic": traffic["cold"] if traffic else None,
+                     "traffic_warm": traffic["warm"] if traffic else None, "traffic_kernel_digest": traffic_rev,
                      "peak_source": "%s bf16 sustained (a seconds-long cuBLAS loop under the power cap); frac_burst is against the "
                                     "burst figure, measured at the SM clock in `clocks`" % peaks["source"],
                      "avg_launch_us": 1e6 * joiner_s / max(st["joiner_launches"], 1),
