@@ -162,8 +162,8 @@ int tw_decode(tw_handle* h, const void* enc, const int32_t* lengths, int32_t B, 
 
 /* Same as tw_decode with HOST buffers: copies the inputs to the device, decodes, copies the four
  * outputs back; synchronises before returning.  For batches decoded in one piece and T >= 16 S the
- * frames are uploaded in three time chunks on a stream of the handle's own (ordered after `stream`)
- * and each chunk is decoded, as a streaming push, while the next one is on its way; the result is
+ * frames are uploaded in two time chunks (the first sixteenth, then the rest) on a stream of the handle's own
+ * (ordered after `stream`) and the first chunk is decoded, as a streaming push, while the second is on its way; the result is
  * the same as tw_decode's.  Pinned host memory is what makes the upload asynchronous.  Must not be
  * called while a streaming session is open on the handle. */
 int tw_decode_host(tw_handle* h, const void* host_enc, const int32_t* host_lengths, int32_t B,

@@ -63,9 +63,9 @@ struct tw_handle {
   char* st_enc = nullptr; int* st_len = nullptr; int* st_tok = nullptr; int* st_lens = nullptr;
   // tw_decode_host uploads the frames in a few time chunks on copy_stream and decodes chunk k (as a streaming
   // session) while chunk k + 1 is still on its way
-  static constexpr int kHostChunks = 3;
+  static constexpr int kHostChunks = 2;
   cudaStream_t copy_stream = nullptr;
-  cudaEvent_t ev_chunk[kHostChunks] = {nullptr, nullptr, nullptr};
+  cudaEvent_t ev_chunk[kHostChunks] = {nullptr, nullptr};
   int* st_chunk_lens = nullptr;                         // [kHostChunks][max_batch]
   double* st_scores = nullptr; int* st_status = nullptr;
 
